@@ -1,0 +1,188 @@
+/*
+ * accerl.h -- C ABI of the int8 Actor policy-inference library for NVIDIA B200 (sm_100a).
+ *
+ * What the library computes.  In the paper's actor-learner loop every Actor runs, per
+ * environment step, one forward pass of the Compressor's quantised policy network on a batch
+ * of states and samples one action per state (Introduction, Fig. 1: the "Agent" share of data
+ * collection; Section 2.1, Overview).  The compressed policy is an int8 post-training-
+ * quantised network whose Conv+ReLU / FC+ReLU pairs are fused into single layers (Section 2.2,
+ * paragraphs "Parameter Quantization" and "Static Computational Graph").  The Corrector later
+ * needs the behaviour probability pi_smaller(a|x) of the action taken (Section 2.3, Eq. V-trace
+ * and Eq. IS).  `accerl_policy_create` takes such a quantised network, `accerl_policy_act`
+ * maps a batch of states to logits, sampled actions and behaviour log-probabilities.
+ *
+ * Arithmetic (fixed; the same on every code path of the library):
+ *   input, frames : x = (float)u / 255.0f;  q = clamp(rintf(x / s_input), -128, 127)
+ *   input, vectors: q = clamp(rintf(obs / s_input), -128, 127)
+ *   contraction   : acc = sum_k w[c,k] * x[k]              int8 x int8 -> int32, zero padding
+ *                   (ACCERL_RELU_IN: x is max(x, 0) first)
+ *   residual      : acc += skip_mul[c] * x_skip[c, y, x]    int32, before the epilogue
+ *   epilogue      : y = fmaf((float)acc, s_in * s_w[c], bias[c]);   s_in * s_w[c] rounded once
+ *                   (ACCERL_RELU_OUT: y = max(y, 0))
+ *                   q = clamp(rintf(y / s_out), -128, 127)   IEEE divide, ties to even
+ *   final layer   : ACCERL_LOGITS stops at y (fp32 logits)
+ *   max-pool      : per-channel max over a kh x kw window, stride `stride`, no padding, floor
+ *   sampling      : logp = z - logsumexp(z);  cdf_i = sum_{j<=i} exp(logp_j);
+ *                   action = first i with u < cdf_i, else A-1;  logp_out = logp[action]
+ *
+ * Conventions.  All sizes are in elements unless they say bytes.  "host" / "device" in a
+ * parameter comment says where the pointer must live.  Nothing is thrown across this ABI and
+ * the library never calls exit/abort: every entry point returns an accerl_status, and
+ * accerl_last_error() gives a message for the calling thread's last failure.  Invalid
+ * arguments are rejected on the host before anything is launched.
+ */
+#ifndef ACCERL_H_
+#define ACCERL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct accerl_policy accerl_policy; /* opaque handle */
+
+typedef enum {
+    ACCERL_OK = 0,
+    ACCERL_ERR_INVALID_ARG = 1,     /* null pointer, bad size, inconsistent layer chain */
+    ACCERL_ERR_UNSUPPORTED = 2,     /* valid description the library has no kernel for */
+    ACCERL_ERR_BATCH_TOO_LARGE = 3, /* batch > max_batch given at create */
+    ACCERL_ERR_OOM = 4,             /* device or host allocation failed */
+    ACCERL_ERR_CUDA = 5,            /* a CUDA runtime / driver call failed */
+    ACCERL_ERR_TIMEOUT = 6          /* a bounded device-side wait gave up (status word set) */
+} accerl_status;
+
+typedef enum { ACCERL_IN_U8_NCHW = 0, ACCERL_IN_F32 = 1 } accerl_input_kind;
+typedef enum { ACCERL_CONV2D = 0, ACCERL_FC = 1, ACCERL_MAXPOOL = 2 } accerl_layer_kind;
+
+/* accerl_layer_desc.flags */
+enum {
+    ACCERL_RELU_IN = 1,  /* apply max(x, 0) to the int8 input before the contraction */
+    ACCERL_RELU_OUT = 2, /* ReLU on the epilogue float, before the clamp */
+    ACCERL_LOGITS = 4    /* last layer: fp32 output, no requantisation */
+};
+
+/* accerl_policy_create flags */
+enum {
+    ACCERL_FLAG_KEEP_ACTIVATIONS = 1, /* give every layer its own output buffer so that
+                                         accerl_policy_read_activation works (parity taps) */
+    ACCERL_FLAG_FORCE_GENERIC = 2     /* use only the plain CUDA-core kernels (no tensor-core
+                                         or fused plans); for cross-checking the fast paths */
+};
+
+/*
+ * One layer.  Conv: input [in_c, in_h, in_w], weights OIHW [out_c][in_c][kh][kw], square
+ * `stride`, symmetric zero `pad`.  FC: in_c = K, out_c = N, in_h = in_w = kh = kw = stride = 1,
+ * pad = 0; an FC fed by a conv/pool output reads it flattened in (C, H, W) order.  Max-pool:
+ * in_c = out_c, kh = kw = window, no weights (w, s_w, bias NULL; s_out must equal s_in).
+ * All pointers are HOST pointers; the library copies what they point to during create and
+ * never keeps them.
+ */
+typedef struct {
+    int32_t kind; /* accerl_layer_kind */
+    uint32_t flags;
+    int32_t in_c, in_h, in_w, out_c, kh, kw, stride, pad;
+    float s_in, s_out;       /* per-tensor activation scales of this layer's input / output */
+    const int8_t *w;         /* host, int8 weights, values in [-127, 127] */
+    const float *s_w;        /* host, [out_c] per-output-channel weight scales */
+    const float *bias;       /* host, [out_c] fp32 */
+    int32_t skip_from;       /* -1, or index of an EARLIER layer whose int8 output (same shape
+                                as this layer's output) is added into the accumulators */
+    const int32_t *skip_mul; /* host, [out_c] integer multipliers, in [0, 32767]; NULL iff
+                                skip_from < 0 */
+} accerl_layer_desc;
+
+/*
+ * Build a policy on CUDA device `device` (Section 2.2: the Compressor hands the Actor a
+ * quantised, fused, static network; this call is the "static graph" step: it validates the
+ * chain, repacks weights into the kernels' layouts, precomputes s_in * s_w[c], allocates the
+ * activation workspace for `max_batch` states and fixes the launch plan).
+ *   out        host, receives the handle (NULL on failure)
+ *   in_kind    ACCERL_IN_U8_NCHW: observations are uint8 [B, C, H, W];
+ *              ACCERL_IN_F32: observations are fp32 [B, D] with in_shape = {D, 1, 1}
+ *   in_shape   host, {C, H, W}
+ *   s_input    scale of the quantised input tensor (must equal layers[0].s_in)
+ *   layers     host, n_layers descriptors; layer i consumes layer i-1's output; the last layer
+ *              must be an FC with ACCERL_LOGITS and out_c = number of actions (1..1024)
+ *   max_batch  largest batch `act` will be called with (>= 1)
+ *   flags      ACCERL_FLAG_* bits
+ * Synchronises the device once; allocates device memory (freed by accerl_policy_destroy).
+ * Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA; *out is NULL then.
+ */
+accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const int32_t in_shape[3],
+                                   float s_input, const accerl_layer_desc *layers,
+                                   int32_t n_layers, int32_t max_batch, uint32_t flags,
+                                   int32_t device);
+
+/*
+ * One Actor step for a batch of states (Introduction, Fig. 1 "Agent"; Section 2.3, Eq. V-trace
+ * for the behaviour log-probability): quantise the observations, run every layer, sample.
+ *   obs_dev       device, uint8 [batch, C, H, W] or fp32 [batch, D]; 16-byte aligned; read only
+ *   uniforms_dev  device, fp32 [batch], each in [0, 1): the random numbers the sampler inverts
+ *   batch         1 .. max_batch
+ *   logits_dev    device, fp32 [batch, A], written
+ *   actions_dev   device, int32 [batch], written; always in [0, A-1]
+ *   logp_dev      device, fp32 [batch], written: log pi(action | state), finite and <= 0
+ *   cuda_stream   a cudaStream_t (NULL = the default stream)
+ * Enqueues kernels on `cuda_stream` and returns without synchronising.  Allocates nothing.
+ * The handle owns the workspace the kernels write, so calls on one handle must not overlap on
+ * the GPU (use one stream per handle, or one handle per stream).  The caller owns all five
+ * buffers.  Errors: INVALID_ARG, BATCH_TOO_LARGE, CUDA (launch failure).
+ */
+accerl_status accerl_policy_act(accerl_policy *p, const void *obs_dev, const float *uniforms_dev,
+                                int32_t batch, float *logits_dev, int32_t *actions_dev,
+                                float *logp_dev, void *cuda_stream);
+
+/*
+ * The same step for callers whose data lives in HOST memory (an Actor process that steps its
+ * environments on the CPU, Section 2.1): copies obs and uniforms to device staging buffers owned
+ * by the handle, runs accerl_policy_act, copies the three results back and waits for them.
+ * All five pointers are host pointers (pinned memory makes the copies asynchronous and faster;
+ * pageable memory works).  The staging buffers are allocated on the first call.  Blocks until
+ * the results are in the host buffers.
+ */
+accerl_status accerl_policy_act_host(accerl_policy *p, const void *obs_host,
+                                     const float *uniforms_host, int32_t batch,
+                                     float *logits_host, int32_t *actions_host, float *logp_host,
+                                     void *cuda_stream);
+
+/*
+ * Parity tap: copy layer `layer`'s int8 output of the most recent `act` call to the host in
+ * canonical NCHW order ([batch, out_c, out_h, out_w]; for FC layers [batch, out_c]).
+ * `layer` = -1 reads the quantised input tensor ([batch, C, H, W] or [batch, D]).
+ * Needs ACCERL_FLAG_KEEP_ACTIVATIONS; synchronises the device.  The final (logits) layer has
+ * no int8 output (INVALID_ARG).  dst_bytes must be at least the tensor's size.
+ */
+accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int32_t batch,
+                                            int8_t *dst_host_nchw, size_t dst_bytes);
+
+/*
+ * Synchronise the stream of the last `act` call and report the device status word: ACCERL_OK,
+ * ACCERL_ERR_TIMEOUT if a kernel's bounded wait gave up, ACCERL_ERR_CUDA for a sticky error.
+ */
+accerl_status accerl_policy_check(accerl_policy *p);
+
+/*
+ * Describe the handle: number of actions, bytes of device workspace, kernel launches per
+ * `act` call and a human-readable plan (one line per launch) written as a NUL-terminated
+ * string into plan_buf (truncated to plan_buf_bytes).  Any output pointer may be NULL.
+ * `batch` selects which plan is described (plans can differ by batch size).
+ */
+accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t *n_actions,
+                                 size_t *workspace_bytes, int32_t *launches_per_act,
+                                 char *plan_buf, size_t plan_buf_bytes);
+
+/* Free the handle and its device memory.  Synchronises the device.  NULL is allowed. */
+void accerl_policy_destroy(accerl_policy *p);
+
+/* Message for the calling thread's most recent failing call; never NULL. */
+const char *accerl_last_error(void);
+
+/* Library version string. */
+const char *accerl_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ACCERL_H_ */
