@@ -1,0 +1,93 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "accerl.h"
+
+namespace accerl {
+
+void set_error(const char *fmt, ...);
+
+#define ACCERL_CUDA_TRY(expr)                                                              \
+    do {                                                                                   \
+        cudaError_t e_ = (expr);                                                           \
+        if (e_ != cudaSuccess) {                                                           \
+            ::accerl::set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e_),    \
+                                __FILE__, __LINE__);                                       \
+            return e_ == cudaErrorMemoryAllocation ? ACCERL_ERR_OOM : ACCERL_ERR_CUDA;     \
+        }                                                                                  \
+    } while (0)
+
+static inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+// One layer as the kernels see it.  Activations live in device memory as NHWC int8 with the
+// channel count padded to a multiple of 4 (`*_cp`), so that four channels form one 32-bit word.
+struct LayerPlan {
+    int kind = 0;
+    uint32_t flags = 0;
+    int in_c = 0, in_h = 0, in_w = 0, out_c = 0, out_h = 0, out_w = 0;
+    int kh = 0, kw = 0, stride = 1, pad = 0;
+    int in_cp = 0, out_cp = 0;
+    float s_in = 1.f, s_out = 1.f;
+    int skip_from = -1;
+    int in_buf = -1, out_buf = -1, skip_buf = -1;  // indices into accerl_policy::bufs
+    // device parameters
+    int32_t *w_generic = nullptr;  // conv: [tap][in_cp/4][oc_pad] words; fc: [oc_pad][K/4]
+    float *kscale = nullptr;       // [oc_pad]  s_in * s_w[c], 0 for padding channels
+    float *bias = nullptr;         // [oc_pad]
+    int32_t *skip_mul = nullptr;   // [oc_pad] or null
+    int oc_pad = 0;                // out_c rounded up to 16
+    std::string how;               // which kernel serves the layer (for accerl_policy_info)
+};
+
+struct DeviceBuf {
+    int8_t *ptr = nullptr;
+    size_t bytes_per_state = 0;
+};
+
+}  // namespace accerl
+
+struct accerl_policy {
+    int device = 0;
+    int in_kind = 0;
+    int in_c = 0, in_h = 0, in_w = 0, in_cp = 0;
+    float s_input = 1.f;
+    int max_batch = 0;
+    uint32_t flags = 0;
+    int n_actions = 0;
+    std::vector<accerl::LayerPlan> layers;
+    std::vector<accerl::DeviceBuf> bufs;  // bufs[0] holds the quantised input
+    int8_t *lut = nullptr;                // device, 256-entry uint8 -> int8 input table
+    int *status_word = nullptr;           // device, set by kernels whose bounded waits give up
+    size_t workspace_bytes = 0;
+    std::vector<void *> owned;            // every device allocation, for destroy
+    cudaStream_t last_stream = nullptr;
+    // host-call staging (allocated on first accerl_policy_act_host)
+    void *st_obs = nullptr;
+    float *st_u = nullptr, *st_logits = nullptr, *st_logp = nullptr;
+    int32_t *st_actions = nullptr;
+};
+
+namespace accerl {
+
+// generic CUDA-core kernels (generic_kernels.cu); every launcher enqueues on `st` and returns
+// the launch status
+cudaError_t launch_ingest_u8(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
+                             int H, int W, int Cp, cudaStream_t st);
+cudaError_t launch_ingest_f32(const float *obs, float s_input, int8_t *out, int B, int D, int Dp,
+                              cudaStream_t st);
+cudaError_t launch_conv_generic(const LayerPlan &L, const int8_t *in, const int8_t *skip,
+                                int8_t *out, int B, cudaStream_t st);
+cudaError_t launch_fc_generic(const LayerPlan &L, const int8_t *in, int8_t *out, float *logits,
+                              int B, cudaStream_t st);
+cudaError_t launch_maxpool_generic(const LayerPlan &L, const int8_t *in, int8_t *out, int B,
+                                   cudaStream_t st);
+cudaError_t launch_sample(const float *logits, const float *u, int B, int A, int32_t *actions,
+                          float *logp, cudaStream_t st);
+
+}  // namespace accerl
