@@ -1,0 +1,184 @@
+"""ctypes binding of libaccerl.so: same names and argument order as include/accerl.h."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB = None
+
+FLAG_KEEP_ACTIVATIONS = 1
+FLAG_FORCE_GENERIC = 2
+RELU_IN, RELU_OUT, LOGITS = 1, 2, 4
+_KINDS = {"conv": 0, "fc": 1, "maxpool": 2}
+STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "BATCH_TOO_LARGE", 4: "OOM", 5: "CUDA",
+          6: "TIMEOUT"}
+
+
+class AccerlError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("accerl %s: %s" % (STATUS.get(status, status), message))
+        self.status = status
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("flags", C.c_uint32),
+                ("in_c", C.c_int32), ("in_h", C.c_int32), ("in_w", C.c_int32),
+                ("out_c", C.c_int32), ("kh", C.c_int32), ("kw", C.c_int32),
+                ("stride", C.c_int32), ("pad", C.c_int32),
+                ("s_in", C.c_float), ("s_out", C.c_float),
+                ("w", C.c_void_p), ("s_w", C.c_void_p), ("bias", C.c_void_p),
+                ("skip_from", C.c_int32), ("skip_mul", C.c_void_p)]
+
+
+def library_path() -> str:
+    return os.path.join(_HERE, "libaccerl.so")
+
+
+def library() -> C.CDLL:
+    """Load libaccerl.so; there is no fallback if it has not been built."""
+    global _LIB
+    if _LIB is None:
+        path = library_path()
+        if not os.path.exists(path):
+            raise ImportError("%s is missing: build it with `python -m paper_2211_15023_b200.build`"
+                              % path)
+        lib = C.CDLL(path)
+        vp, i32, f32 = C.c_void_p, C.c_int32, C.c_float
+        lib.accerl_policy_create.argtypes = [C.POINTER(vp), i32, C.POINTER(i32), f32,
+                                             C.POINTER(LayerDesc), i32, i32, C.c_uint32, i32]
+        lib.accerl_policy_act.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
+        lib.accerl_policy_act_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
+        lib.accerl_policy_read_activation.argtypes = [vp, i32, i32, vp, C.c_size_t]
+        lib.accerl_policy_check.argtypes = [vp]
+        lib.accerl_policy_info.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_size_t),
+                                           C.POINTER(i32), C.c_char_p, C.c_size_t]
+        lib.accerl_policy_destroy.argtypes = [vp]
+        lib.accerl_policy_destroy.restype = None
+        lib.accerl_last_error.restype = C.c_char_p
+        lib.accerl_version.restype = C.c_char_p
+        for f in ("create", "act", "act_host", "read_activation", "check", "info"):
+            getattr(lib, "accerl_policy_" + f).restype = C.c_int
+        _LIB = lib
+    return _LIB
+
+
+def _check(status: int):
+    if status != 0:
+        raise AccerlError(status, library().accerl_last_error().decode())
+
+
+def _out_hw(l):
+    if l["kind"] == "fc":
+        return 1, 1
+    return ((l["in_h"] + 2 * l["pad"] - l["kh"]) // l["stride"] + 1,
+            (l["in_w"] + 2 * l["pad"] - l["kw"]) // l["stride"] + 1)
+
+
+class Policy:
+    """An int8 policy resident on one GPU.
+
+    ``policy`` is a dict with ``in_kind`` ("u8" | "f32"), ``in_shape`` (C, H, W),
+    ``s_input`` and ``layers``: dicts with kind, in_c, in_h, in_w, out_c, kh, kw, stride, pad,
+    relu_in, relu_out, logits, skip_from, s_in, s_out and numpy arrays w (int8 OIHW), s_w, bias,
+    skip_mul (or None).
+    """
+
+    def __init__(self, policy: dict, max_batch: int, flags: int = 0, device: int = 0):
+        lib = library()
+        self._h = C.c_void_p()
+        self.layers = policy["layers"]
+        n = len(self.layers)
+        descs = (LayerDesc * n)()
+        keep = []  # host arrays must outlive the create call only
+        for i, l in enumerate(self.layers):
+            d = descs[i]
+            d.kind = _KINDS[l["kind"]]
+            d.flags = (RELU_IN if l["relu_in"] else 0) | (RELU_OUT if l["relu_out"] else 0) | \
+                (LOGITS if l["logits"] else 0)
+            for k in ("in_c", "in_h", "in_w", "out_c", "kh", "kw", "stride", "pad", "skip_from"):
+                setattr(d, k, int(l[k]))
+            d.s_in, d.s_out = float(l["s_in"]), float(l["s_out"])
+            for k, dt in (("w", np.int8), ("s_w", np.float32), ("bias", np.float32),
+                          ("skip_mul", np.int32)):
+                if l.get(k) is not None:
+                    a = np.ascontiguousarray(l[k], dt)
+                    keep.append(a)
+                    setattr(d, k, a.ctypes.data)
+        shape = (C.c_int32 * 3)(*[int(v) for v in policy["in_shape"]])
+        self.in_kind = policy["in_kind"]
+        self.in_shape = tuple(int(v) for v in policy["in_shape"])
+        self.max_batch = int(max_batch)
+        self.device = int(device)
+        _check(lib.accerl_policy_create(C.byref(self._h), 0 if self.in_kind == "u8" else 1, shape,
+                                        float(policy["s_input"]), descs, n, self.max_batch,
+                                        int(flags), self.device))
+        self.n_actions = int(self.layers[-1]["out_c"])
+
+    # -- the hot call ---------------------------------------------------------------------
+    def act(self, obs, uniforms, out=None, stream=None):
+        """obs, uniforms: CUDA torch tensors.  Returns (logits, actions, logp) CUDA tensors."""
+        import torch
+        b = int(obs.shape[0])
+        if out is None:
+            dev = obs.device
+            out = (torch.empty((b, self.n_actions), dtype=torch.float32, device=dev),
+                   torch.empty(b, dtype=torch.int32, device=dev),
+                   torch.empty(b, dtype=torch.float32, device=dev))
+        if stream is None:
+            stream = torch.cuda.current_stream(obs.device).cuda_stream
+        assert obs.is_contiguous() and uniforms.is_contiguous() and obs.is_cuda and uniforms.is_cuda
+        assert obs.dtype == (torch.uint8 if self.in_kind == "u8" else torch.float32)
+        assert uniforms.dtype == torch.float32 and uniforms.numel() == b
+        _check(library().accerl_policy_act(self._h, obs.data_ptr(), uniforms.data_ptr(), b,
+                                           out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(),
+                                           stream))
+        return out
+
+    def act_raw(self, obs_ptr, u_ptr, batch, logits_ptr, actions_ptr, logp_ptr, stream=0) -> int:
+        """Unchecked pass-through returning the status code (for ABI tests)."""
+        return library().accerl_policy_act(self._h, obs_ptr, u_ptr, batch, logits_ptr, actions_ptr,
+                                           logp_ptr, stream)
+
+    def act_host(self, obs, uniforms, out, stream=0):
+        """obs, uniforms, out=(logits, actions, logp): host tensors/arrays (pinned is faster)."""
+        ptr = lambda a: a.data_ptr() if hasattr(a, "data_ptr") else a.ctypes.data  # noqa: E731
+        _check(library().accerl_policy_act_host(self._h, ptr(obs), ptr(uniforms), int(obs.shape[0]),
+                                                ptr(out[0]), ptr(out[1]), ptr(out[2]), stream))
+        return out
+
+    # -- parity taps and introspection --------------------------------------------------------
+    def read_activation(self, layer: int, batch: int) -> np.ndarray:
+        if layer < 0:
+            shape = (batch,) + self.in_shape
+        else:
+            l = self.layers[layer]
+            shape = (batch, l["out_c"]) + _out_hw(l)
+        dst = np.empty(shape, np.int8)
+        _check(library().accerl_policy_read_activation(self._h, layer, batch, dst.ctypes.data,
+                                                       dst.nbytes))
+        return dst
+
+    def check(self):
+        _check(library().accerl_policy_check(self._h))
+
+    def info(self, batch: int | None = None) -> dict:
+        na, ws, nl = C.c_int32(), C.c_size_t(), C.c_int32()
+        buf = C.create_string_buffer(1 << 16)
+        _check(library().accerl_policy_info(self._h, batch or self.max_batch, C.byref(na),
+                                            C.byref(ws), C.byref(nl), buf, len(buf)))
+        return dict(n_actions=na.value, workspace_bytes=ws.value, launches_per_act=nl.value,
+                    plan=buf.value.decode())
+
+    def close(self):
+        if self._h:
+            library().accerl_policy_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
