@@ -1,0 +1,163 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as W
+from parity_util import calibrated, compare
+
+pytestmark = pytest.mark.gpu
+
+SMALL = {  # name -> batches that span several tiles plus ragged tails
+    "cartpole_mlp": [1, 3, 127, 160],
+    "lunarlander_mlp": [129, 4096],
+    "nature_cnn_b160": [1, 3, 37],
+    "student_cnn_b8192": [5, 33],
+    "impala_resnet_b16384": [2, 9],
+}
+
+
+def _run(pol, obs, u, flags, max_batch=None):
+    import paper_2211_15023_b200 as P
+    g = P.Policy(pol, max_batch or obs.shape[0], flags=flags)
+    out = g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())
+    torch.cuda.synchronize()
+    g.check()
+    return g, [t.cpu().numpy() for t in out]
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+@pytest.mark.parametrize("flags", [1, 3], ids=["default_plan", "generic_plan"])
+def test_small_batches_every_activation(name, flags):
+    pol = calibrated(name)
+    for b in SMALL[name]:
+        obs, u = W.observations(name, b), W.uniforms(name, b)
+        ref = oracle.forward(pol, obs, u)
+        g, (logits, actions, logp) = _run(pol, obs, u, flags)
+        stats = compare(ref, logits, actions, logp, taps=g.read_activation)
+        assert stats["int8_mismatch"] == 0
+        # three runs must give identical bytes (races show up as nondeterminism)
+        for _ in range(2):
+            out2 = g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())
+            assert np.array_equal(out2[0].cpu().numpy(), logits)
+            assert np.array_equal(out2[1].cpu().numpy(), actions)
+        g.close()
+
+
+FULL = ["cartpole_mlp", "lunarlander_mlp", "nature_cnn_b160", "nature_cnn_b8192",
+        "student_cnn_b8192", "impala_resnet_b16384"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_batch_sampled_states(name):
+    """Full batch, no taps flag (the plan the benchmark times); the oracle checks a sample."""
+    import paper_2211_15023_b200 as P
+    pol = calibrated(name)
+    b = W.config(name)["batch"]
+    obs, u = W.observations(name, b), W.uniforms(name, b)
+    g = P.Policy(pol, b, flags=0)
+    out = g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())
+    torch.cuda.synchronize()
+    g.check()
+    logits, actions, logp = [t.cpu().numpy() for t in out]
+    rng = np.random.default_rng(99)
+    n = min(b, 48)
+    idx = np.unique(np.concatenate([[0, b - 1], rng.choice(b, n, replace=False)]))
+    ref = oracle.forward(pol, obs[idx], u[idx], keep=False)
+    compare(ref, logits[idx], actions[idx], logp[idx])
+    assert np.all((actions >= 0) & (actions < logits.shape[1]))
+    assert np.all(np.isfinite(logp)) and np.all(logp <= 0) and np.all(np.isfinite(logits))
+    # the same states alone in a small batch give the same bytes (no cross-state coupling)
+    small = g.act(torch.from_numpy(obs[idx[:7]]).cuda(), torch.from_numpy(u[idx[:7]]).cuda())
+    assert np.array_equal(small[0].cpu().numpy(), logits[idx[:7]])
+    assert np.array_equal(small[1].cpu().numpy(), actions[idx[:7]])
+    g.close()
+
+
+def test_act_host_matches_device_call():
+    import paper_2211_15023_b200 as P
+    name = "nature_cnn_b160"
+    pol = calibrated(name)
+    obs, u = W.observations(name, 20), W.uniforms(name, 20)
+    g = P.Policy(pol, 32)
+    dev = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+    host = (torch.empty((20, 18), dtype=torch.float32).pin_memory(),
+            torch.empty(20, dtype=torch.int32).pin_memory(),
+            torch.empty(20, dtype=torch.float32).pin_memory())
+    g.act_host(torch.from_numpy(obs).pin_memory(), torch.from_numpy(u).pin_memory(), host)
+    for a, b in zip(dev, host):
+        assert np.array_equal(a, b.numpy())
+    g.close()
+
+
+def test_saturating_inputs_and_extreme_uniforms():
+    import paper_2211_15023_b200 as P
+    name = "lunarlander_mlp"
+    pol = calibrated(name)
+    obs = (W.observations(name, 64) * 5).astype(np.float32)   # far outside the calibrated range
+    u = np.concatenate([np.zeros(32), np.full(32, np.nextafter(np.float32(1), np.float32(0)))]
+                       ).astype(np.float32)
+    ref = oracle.forward(pol, obs, u)
+    g = P.Policy(pol, 64, flags=1)
+    out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+    compare(ref, *out, taps=g.read_activation)
+    g.close()
+
+
+def test_many_actions_wide_sampler():
+    # 40 actions exercise the sampler that strides a warp over the row
+    import paper_2211_15023_b200 as P
+    rng = np.random.default_rng(5)
+    layers = W.mlp([6, 32, 40])
+    params = [dict(w=rng.standard_normal((l["out_c"], l["in_c"], 1, 1)).astype(np.float32),
+                   bias=rng.standard_normal(l["out_c"]).astype(np.float32) * 0.1) for l in layers]
+    calib = rng.standard_normal((256, 6)).astype(np.float32)
+    pol = oracle.calibrate("f32", (6, 1, 1), layers, params, calib)
+    obs = rng.standard_normal((77, 6)).astype(np.float32)
+    u = rng.random(77, dtype=np.float32)
+    ref = oracle.forward(pol, obs, u)
+    g = P.Policy(pol, 77, flags=1)
+    out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+    compare(ref, *out, taps=g.read_activation)
+    g.close()
+
+
+def test_odd_shapes_padding_stride_pool_residual():
+    import paper_2211_15023_b200 as P
+    rng = np.random.default_rng(11)
+    layers = [W._conv(3, 11, 9, 5, 3, 2, 1, relu_out=False), W._pool(5, 6, 5, 3, 2),
+              W._conv(5, 2, 2, 5, 3, 1, 1, relu_in=True),
+              W._conv(5, 2, 2, 5, 3, 1, 1, relu_out=False, skip_from=1),
+              W._fc(20, 7, relu_in=True), W._fc(7, 3, relu_out=False, logits=True)]
+    params = [None if l["kind"] == "maxpool" else
+              dict(w=rng.standard_normal((l["out_c"], l["in_c"], l["kh"], l["kw"])
+                                         ).astype(np.float32) * 0.3,
+                   bias=rng.standard_normal(l["out_c"]).astype(np.float32) * 0.1) for l in layers]
+    calib = rng.integers(0, 256, (16, 3, 11, 9), dtype=np.uint8)
+    pol = oracle.calibrate("u8", (3, 11, 9), layers, params, calib)
+    obs = rng.integers(0, 256, (13, 3, 11, 9), dtype=np.uint8)
+    u = rng.random(13, dtype=np.float32)
+    ref = oracle.forward(pol, obs, u)
+    g = P.Policy(pol, 13, flags=1)
+    out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+    compare(ref, *out, taps=g.read_activation)
+    g.close()
+
+
+def test_abi_rejects_bad_calls_without_launching():
+    import paper_2211_15023_b200 as P
+    pol = calibrated("cartpole_mlp")
+    g = P.Policy(pol, 8)
+    obs = torch.zeros((16, 4), device="cuda")
+    u = torch.zeros(16, device="cuda")
+    lo, ac, lp = (torch.empty((16, 2), device="cuda"), torch.empty(16, dtype=torch.int32, device="cuda"),
+                  torch.empty(16, device="cuda"))
+    assert g.act_raw(obs.data_ptr(), u.data_ptr(), 16, lo.data_ptr(), ac.data_ptr(), lp.data_ptr()) == 3
+    assert g.act_raw(obs.data_ptr(), u.data_ptr(), 0, lo.data_ptr(), ac.data_ptr(), lp.data_ptr()) == 1
+    assert g.act_raw(None, u.data_ptr(), 4, lo.data_ptr(), ac.data_ptr(), lp.data_ptr()) == 1
+    assert g.act_raw(obs.data_ptr() + 4, u.data_ptr(), 4, lo.data_ptr(), ac.data_ptr(), lp.data_ptr()) == 1
+    with pytest.raises(P.AccerlError):
+        g.read_activation(0, 4)          # no KEEP_ACTIVATIONS flag
+    g.check()
+    g.close()
