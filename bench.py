@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the int8 Actor policy-inference path: states/s on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload NAME]
+
+A step is one `accerl_policy_act` call: input quantisation, every layer of the network and
+the sampler, on one batch of synthetic states.  The default workload is the Nature-CNN policy
+(the paper's "Original" network of the table "network architecture and inference time") at
+batch 8192; the other workloads are timed briefly and reported under "other_workloads".
+With N > 1 (torchrun) every rank runs the same batch size on its own GPU (states are
+independent, there is no exchange step) and the time is the maximum over ranks.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+METRIC = "int8 policy-inference states/sec"
+UNIT = "states/s"
+DEFAULT_WORKLOAD = "nature_cnn_b8192"
+OUT_BYTES = lambda a: 4 * a + 8          # noqa: E731  logits + action + logp per state
+
+
+def peaks() -> dict:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows, self.proc, self.index = [], None, index
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([t.strip() for t in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self) -> dict:
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        busy = [v for v in sm if v >= 0.5 * max(sm)]
+        return dict(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+def algorithmic(name: str, batch: int) -> dict:
+    """Algorithmic work of one step: 2 x MACs, and input + output bytes per state."""
+    a = W.n_actions(name)
+    return dict(ops=2 * W.macs_per_state(name) * batch,
+                bytes=(W.input_bytes_per_state(name) + 4 + OUT_BYTES(a)) * batch)
+
+
+def launch_work(name: str, plan: str, batch: int) -> list:
+    """Per launch of the plan: kernel name, int8 ops (2 x MACs) and algorithmic bytes."""
+    c = W.config(name)
+    layers = c["layers"]
+    a = W.n_actions(name)
+
+    def tensor_bytes(i):  # int8 output of layer i, or the quantised input for i = -1
+        if i < 0:
+            return int(np.prod(c["in_shape"]))
+        oh, ow = W.out_hw(layers[i])
+        return layers[i]["out_c"] * oh * ow
+
+    out = []
+    for line in plan.strip().splitlines():
+        head, rest = line.split(" covers ", 1)
+        kernel = head.split(": ", 1)[1]
+        covers = rest.split(" (")[0]
+        ops, nbytes, first_in, last_out = 0, 0, None, None
+        for part in covers.split("+"):
+            part = part.strip()
+            if part == "ingest":
+                nbytes += W.input_bytes_per_state(name)
+                last_out = -1
+            elif part == "sample":
+                nbytes += 4 + 8  # uniform in, action + logp out (logits counted with their layer)
+            else:
+                idx = part.replace("layers", "").replace("layer", "").strip()
+                lo, hi = (int(t) for t in idx.split("-")) if "-" in idx else (int(idx), int(idx))
+                for i in range(lo, hi + 1):
+                    l = layers[i]
+                    if l["kind"] != "maxpool":
+                        oh, ow = W.out_hw(l)
+                        ops += 2 * oh * ow * l["out_c"] * l["in_c"] * l["kh"] * l["kw"]
+                        if l["skip_from"] >= 0 and not (lo <= l["skip_from"] <= hi):
+                            nbytes += tensor_bytes(l["skip_from"])
+                if first_in is None and last_out is None:
+                    first_in = lo - 1
+                last_out = hi
+        if first_in is not None:
+            nbytes += tensor_bytes(first_in)
+        if last_out is not None:
+            nbytes += 4 * a if last_out == len(layers) - 1 else tensor_bytes(last_out)
+        out.append(dict(kernel=kernel, covers=covers, ops=ops * batch, bytes=nbytes * batch))
+    return out
+
+
+def run_reference(args) -> None:
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    name = args.workload
+    pol = W.drawn_int8_policy(name)
+    sample = min(W.config(name)["batch"], args.ref_sample)
+    obs, u = W.observations(name, sample), W.uniforms(name, sample)
+    for _ in range(args.warmup):
+        oracle.forward(pol, obs, u, keep=False)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.forward(pol, obs, u, keep=False)
+    dt = (time.perf_counter() - t0) / args.steps
+    cores = os.cpu_count()
+    v = sample / dt
+    desc = "%d states of %s per step (oracle/accerl_oracle.c, OpenMP over states)" % (sample, name)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic", "config": {"workload": name, "batch": sample},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def time_workload(P, torch, name, batch, steps, warmup, n_buffers, device, dist=None, clocks=False):
+    """Times `steps` act calls with CUDA events on the launching stream; returns a dict."""
+    pol = W.drawn_int8_policy(name)
+    g = P.Policy(pol, batch, device=device)
+    a = g.n_actions
+    obs_np = W.observations(name, batch)
+    # distinct device copies of the input so that consecutive steps never re-read warm lines
+    obs = [torch.from_numpy(np.roll(obs_np, i, axis=0)).to("cuda:%d" % device) for i in range(n_buffers)]
+    u = torch.from_numpy(W.uniforms(name, batch)).to("cuda:%d" % device)
+    out = (torch.empty((batch, a), dtype=torch.float32, device=u.device),
+           torch.empty(batch, dtype=torch.int32, device=u.device),
+           torch.empty(batch, dtype=torch.float32, device=u.device))
+    stream = torch.cuda.current_stream(u.device)
+    for i in range(warmup):
+        g.act(obs[i % n_buffers], u, out, stream.cuda_stream)
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+        torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(device) if clocks else None
+    if sampler:
+        sampler.__enter__()
+        time.sleep(0.25)
+    ev0.record(stream)
+    for i in range(steps):
+        g.act(obs[i % n_buffers], u, out, stream.cuda_stream)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    if sampler:
+        time.sleep(0.15)
+        sampler.__exit__()
+    ms = ev0.elapsed_time(ev1) / steps
+    if dist is not None:
+        t = torch.tensor([ms], device=u.device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        ms = float(t.item())
+    g.check()
+    info = g.info()
+    # per-launch device times (a second pass over the same steps with events around each launch)
+    per = np.zeros(info["launches_per_act"], np.float64)
+    for i in range(steps):
+        per += g.act_timed(obs[i % n_buffers], u, out, stream.cuda_stream)
+    per /= steps
+    res = dict(ms=ms, info=info, per_launch_ms=per, policy=g, obs=obs_np, u=u, out=out,
+               clocks=sampler.summary() if sampler else None)
+    return res
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(W.CONFIGS))
+    ap.add_argument("--ref-sample", type=int, default=256)
+    ap.add_argument("--cpu-sample", type=int, default=512)
+    ap.add_argument("--no-others", action="store_true", help="skip the brief runs of other workloads")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2211_15023_b200 as P
+    P.library()  # fails loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+
+    name = args.workload
+    batch = W.config(name)["batch"]
+    in_bytes = W.input_bytes_per_state(name) * batch
+    n_buffers = 3 if in_bytes * 3 < (8 << 30) else 2
+    r = time_workload(P, torch, name, batch, args.steps, args.warmup, n_buffers, local, dist,
+                      clocks=(rank == 0))
+    ms = r["ms"]
+    g = r["policy"]
+    clocks = r["clocks"]
+    value = batch * world / (ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point (pinned memory, copies timed)
+    a = g.n_actions
+    obs_pin = torch.from_numpy(r["obs"]).pin_memory()
+    u_pin = r["u"].cpu().pin_memory()
+    out_pin = (torch.empty((batch, a), dtype=torch.float32).pin_memory(),
+               torch.empty(batch, dtype=torch.int32).pin_memory(),
+               torch.empty(batch, dtype=torch.float32).pin_memory())
+    stream = torch.cuda.current_stream()
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(3):
+        g.act_host(obs_pin, u_pin, out_pin, stream.cuda_stream)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(e2e_steps):
+        g.act_host(obs_pin, u_pin, out_pin, stream.cuda_stream)
+    ev1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (largest share of the per-launch device time)
+    pk = peaks()
+    work = launch_work(name, r["info"]["plan"], batch)
+    per = r["per_launch_ms"]
+    top = int(np.argmax(per))
+    int8_peak = 2.0 * pk["bf16_tflops"]  # dense int8 = 2 x dense bf16 (nominal ratio) x measured
+    t_tensor = work[top]["ops"] / (int8_peak * 1e12)
+    t_hbm = work[top]["bytes"] / (pk["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm:
+        achieved = work[top]["ops"] / (per[top] * 1e-3) / 1e12
+        roof = dict(bound="tensor", achieved=achieved, peak=int8_peak, unit="TOP/s",
+                    frac=achieved / int8_peak)
+    else:
+        achieved = work[top]["bytes"] / (per[top] * 1e-3) / 1e9
+        roof = dict(bound="hbm", achieved=achieved, peak=pk["hbm_gbs"], unit="GB/s",
+                    frac=achieved / pk["hbm_gbs"])
+    roof.update(traffic=None, kernel=work[top]["kernel"], covers=work[top]["covers"],
+                kernel_ms=float(per[top]), share=float(per[top] / per.sum()),
+                peak_source="%s (int8 = 2 x bf16 burst)" % pk["source"] if roof["bound"] == "tensor"
+                else pk["source"])
+    whole = algorithmic(name, batch)
+    step_floor_ms = max(whole["ops"] / (int8_peak * 1e12), whole["bytes"] / (pk["hbm_gbs"] * 1e9)) * 1e3
+    launches = [dict(kernel=w["kernel"], covers=w["covers"], ms=float(m)) for w, m in zip(work, per)]
+
+    # ---- the other workloads, briefly (kernel-resident timing only)
+    others = {}
+    if not args.no_others and world == 1:
+        del r
+        g.close()
+        for other in W.CONFIGS:
+            if other == name:
+                continue
+            ob = W.config(other)["batch"]
+            nb = 3 if W.input_bytes_per_state(other) * ob * 3 < (8 << 30) else 2
+            o = time_workload(P, torch, other, ob, max(5, args.steps // 2), 3, nb, local)
+            w = algorithmic(other, ob)
+            floor = max(w["ops"] / (int8_peak * 1e12), w["bytes"] / (pk["hbm_gbs"] * 1e9)) * 1e3
+            others[other] = dict(batch=ob, ms_per_step=o["ms"], states_per_s=ob / (o["ms"] * 1e-3),
+                                 launches=o["info"]["launches_per_act"],
+                                 frac_of_step_roofline=floor / o["ms"])
+            o["policy"].close()
+
+    # ---- CPU oracle on a bounded sample of the same workload (reported baseline)
+    import oracle
+    sample = min(batch, args.cpu_sample)
+    pol = W.drawn_int8_policy(name)
+    so, su = W.observations(name, sample), W.uniforms(name, sample)
+    oracle.forward(pol, so[:8], su[:8], keep=False)
+    t0 = time.perf_counter()
+    oracle.forward(pol, so, su, keep=False)
+    cpu_dt = time.perf_counter() - t0
+    cpu = dict(value=sample / cpu_dt, unit=UNIT, cores=os.cpu_count(), kind="oracle",
+               sample="first %d states of the %d-state batch, one pass" % (sample, batch))
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": name, "batch_per_gpu": batch,
+                   "l2": "inputs larger than L2: %d input buffers of %.0f MB rotate" %
+                         (n_buffers, in_bytes / 1e6),
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks,
+        "e2e": {"value": batch * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": in_bytes + 4 * batch,
+                "d2h_bytes_per_step": OUT_BYTES(a) * batch},
+        "gpu_launches": int(len(per) * args.steps),
+        "roofline": roof,
+        "step_roofline": {"floor_ms": step_floor_ms, "frac": step_floor_ms / ms,
+                          "ops_per_state": whole["ops"] // batch,
+                          "bytes_per_state": whole["bytes"] // batch},
+        "launches": launches,
+        "cpu_baseline": cpu,
+        "other_workloads": others,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -135,6 +135,19 @@ accerl_status accerl_policy_act(accerl_policy *p, const void *obs_dev, const flo
                                 float *logp_dev, void *cuda_stream);
 
 /*
+ * accerl_policy_act with a stopwatch on every kernel launch, for measuring where the Actor's
+ * inference time goes (the paper's own method in the Introduction, Fig. 1, one level down):
+ * records CUDA events on `cuda_stream` around each launch of the plan, runs the step, waits for
+ * it and writes the device time of launch i (milliseconds) to launch_ms_host[i].  The order is
+ * that of accerl_policy_info's plan lines; launch_ms_len must be >= launches_per_act.  The
+ * events are created on the first call.  Blocks until the step has finished.
+ */
+accerl_status accerl_policy_act_timed(accerl_policy *p, const void *obs_dev,
+                                      const float *uniforms_dev, int32_t batch, float *logits_dev,
+                                      int32_t *actions_dev, float *logp_dev, void *cuda_stream,
+                                      float *launch_ms_host, int32_t launch_ms_len);
+
+/*
  * The same step for callers whose data lives in HOST memory (an Actor process that steps its
  * environments on the CPU, Section 2.1): copies obs and uniforms to device staging buffers owned
  * by the handle, runs accerl_policy_act, copies the three results back and waits for them.

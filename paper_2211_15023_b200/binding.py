@@ -50,6 +50,7 @@ def library() -> C.CDLL:
         lib.accerl_policy_create.argtypes = [C.POINTER(vp), i32, C.POINTER(i32), f32,
                                              C.POINTER(LayerDesc), i32, i32, C.c_uint32, i32]
         lib.accerl_policy_act.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
+        lib.accerl_policy_act_timed.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, i32]
         lib.accerl_policy_act_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
         lib.accerl_policy_read_activation.argtypes = [vp, i32, i32, vp, C.c_size_t]
         lib.accerl_policy_check.argtypes = [vp]
@@ -59,7 +60,7 @@ def library() -> C.CDLL:
         lib.accerl_policy_destroy.restype = None
         lib.accerl_last_error.restype = C.c_char_p
         lib.accerl_version.restype = C.c_char_p
-        for f in ("create", "act", "act_host", "read_activation", "check", "info"):
+        for f in ("create", "act", "act_timed", "act_host", "read_activation", "check", "info"):
             getattr(lib, "accerl_policy_" + f).restype = C.c_int
         _LIB = lib
     return _LIB
@@ -136,6 +137,19 @@ class Policy:
                                            out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(),
                                            stream))
         return out
+
+    def act_timed(self, obs, uniforms, out, stream=None) -> np.ndarray:
+        """One step with CUDA events around every launch; returns milliseconds per launch."""
+        import torch
+        if stream is None:
+            stream = torch.cuda.current_stream(obs.device).cuda_stream
+        n = self.info()["launches_per_act"]
+        ms = np.zeros(n, np.float32)
+        _check(library().accerl_policy_act_timed(self._h, obs.data_ptr(), uniforms.data_ptr(),
+                                                 int(obs.shape[0]), out[0].data_ptr(),
+                                                 out[1].data_ptr(), out[2].data_ptr(), stream,
+                                                 ms.ctypes.data, n))
+        return ms
 
     def act_raw(self, obs_ptr, u_ptr, batch, logits_ptr, actions_ptr, logp_ptr, stream=0) -> int:
         """Unchecked pass-through returning the status code (for ABI tests)."""

@@ -208,6 +208,74 @@ void pack_generic(const accerl_layer_desc &d, LayerPlan &L, std::vector<int32_t>
 
 using namespace accerl;
 
+// argument checks shared by the act entry points (nothing is launched when they fail)
+static accerl_status check_act_args(accerl_policy *p, const void *obs_dev,
+                                    const float *uniforms_dev, int32_t batch, float *logits_dev,
+                                    int32_t *actions_dev, float *logp_dev)
+{
+    if (!p || !obs_dev || !uniforms_dev || !logits_dev || !actions_dev || !logp_dev) {
+        set_error("act: null argument");
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    if (batch < 1) {
+        set_error("act: batch must be at least 1");
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    if (batch > p->max_batch) {
+        set_error("act: batch %d exceeds max_batch %d", batch, p->max_batch);
+        return ACCERL_ERR_BATCH_TOO_LARGE;
+    }
+    if (((uintptr_t)obs_dev & 15) || ((uintptr_t)uniforms_dev & 3) || ((uintptr_t)logits_dev & 3) ||
+        ((uintptr_t)actions_dev & 3) || ((uintptr_t)logp_dev & 3)) {
+        set_error("act: misaligned pointer (obs needs 16 bytes, the others 4)");
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    return ACCERL_OK;
+}
+
+// Enqueue the plan's launches; with `ev`, record ev[i] before launch i and ev[n] after the last.
+static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const float *uniforms_dev,
+                               int B, float *logits_dev, int32_t *actions_dev, float *logp_dev,
+                               cudaStream_t st, cudaEvent_t *ev)
+{
+    p->last_stream = st;
+    for (size_t i = 0; i < p->steps.size(); ++i) {
+        const Step &s = p->steps[i];
+        if (ev) ACCERL_CUDA_TRY(cudaEventRecord(ev[i], st));
+        const LayerPlan *L = s.layer >= 0 ? &p->layers[s.layer] : nullptr;
+        const int8_t *in = L ? p->bufs[L->in_buf].ptr : nullptr;
+        int8_t *o = L && L->out_buf >= 0 ? p->bufs[L->out_buf].ptr : nullptr;
+        switch (s.kind) {
+        case Step::INGEST: {
+            int8_t *x = p->bufs[p->layers[0].in_buf].ptr;
+            if (p->in_kind == ACCERL_IN_U8_NCHW)
+                ACCERL_CUDA_TRY(launch_ingest_u8((const uint8_t *)obs_dev, p->lut, x, B, p->in_c,
+                                                 p->in_h, p->in_w, p->in_cp, st));
+            else
+                ACCERL_CUDA_TRY(launch_ingest_f32((const float *)obs_dev, p->s_input, x, B, p->in_c,
+                                                  p->in_cp, st));
+            break;
+        }
+        case Step::CONV_GENERIC:
+            ACCERL_CUDA_TRY(launch_conv_generic(
+                *L, in, L->skip_buf >= 0 ? p->bufs[L->skip_buf].ptr : nullptr, o, B, st));
+            break;
+        case Step::FC_GENERIC:
+            ACCERL_CUDA_TRY(launch_fc_generic(*L, in, o, logits_dev, B, st));
+            break;
+        case Step::POOL_GENERIC:
+            ACCERL_CUDA_TRY(launch_maxpool_generic(*L, in, o, B, st));
+            break;
+        case Step::SAMPLE:
+            ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev,
+                                          logp_dev, st));
+            break;
+        }
+    }
+    if (ev) ACCERL_CUDA_TRY(cudaEventRecord(ev[p->steps.size()], st));
+    return ACCERL_OK;
+}
+
 extern "C" {
 
 const char *accerl_last_error(void) { return g_err; }
@@ -219,6 +287,7 @@ void accerl_policy_destroy(accerl_policy *p)
     DeviceGuard g(p->device);
     cudaDeviceSynchronize();
     for (void *d : p->owned) cudaFree(d);
+    for (cudaEvent_t ev : p->events) cudaEventDestroy(ev);
     delete p;
 }
 
@@ -412,6 +481,29 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         std::vector<int> zero(4, 0);
         if ((st = upload(p, zero, &p->status_word)) != ACCERL_OK) return fail(st);
     }
+    // ---- launch plan
+    {
+        Step s0;
+        s0.kind = Step::INGEST;
+        s0.kernel = in_kind == ACCERL_IN_U8_NCHW ? "ingest_u8_kernel" : "ingest_f32_kernel";
+        s0.covers = "ingest";
+        p->steps.push_back(s0);
+        for (int i = 0; i < n_layers; ++i) {
+            Step s;
+            s.layer = i;
+            s.kind = p->layers[i].kind == ACCERL_CONV2D ? Step::CONV_GENERIC
+                     : p->layers[i].kind == ACCERL_FC   ? Step::FC_GENERIC
+                                                        : Step::POOL_GENERIC;
+            s.kernel = p->layers[i].how;
+            s.covers = "layer " + std::to_string(i);
+            p->steps.push_back(s);
+        }
+        Step ss;
+        ss.kind = Step::SAMPLE;
+        ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
+        ss.covers = "sample";
+        p->steps.push_back(ss);
+    }
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         set_error("create: %s", cudaGetErrorString(e));
@@ -425,48 +517,39 @@ accerl_status accerl_policy_act(accerl_policy *p, const void *obs_dev, const flo
                                 int32_t batch, float *logits_dev, int32_t *actions_dev,
                                 float *logp_dev, void *cuda_stream)
 {
-    if (!p || !obs_dev || !uniforms_dev || !logits_dev || !actions_dev || !logp_dev) {
-        set_error("act: null argument");
-        return ACCERL_ERR_INVALID_ARG;
-    }
-    if (batch < 1) {
-        set_error("act: batch must be at least 1");
-        return ACCERL_ERR_INVALID_ARG;
-    }
-    if (batch > p->max_batch) {
-        set_error("act: batch %d exceeds max_batch %d", batch, p->max_batch);
-        return ACCERL_ERR_BATCH_TOO_LARGE;
-    }
-    if (((uintptr_t)obs_dev & 15) || ((uintptr_t)uniforms_dev & 3) || ((uintptr_t)logits_dev & 3) ||
-        ((uintptr_t)actions_dev & 3) || ((uintptr_t)logp_dev & 3)) {
-        set_error("act: misaligned pointer (obs needs 16 bytes, the others 4)");
-        return ACCERL_ERR_INVALID_ARG;
-    }
+    accerl_status v = check_act_args(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev,
+                                     logp_dev);
+    if (v != ACCERL_OK) return v;
     DeviceGuard guard(p->device);
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    p->last_stream = st;
-    const int B = batch;
-    int8_t *x = p->bufs[p->layers[0].in_buf].ptr;
-    if (p->in_kind == ACCERL_IN_U8_NCHW)
-        ACCERL_CUDA_TRY(launch_ingest_u8((const uint8_t *)obs_dev, p->lut, x, B, p->in_c, p->in_h,
-                                         p->in_w, p->in_cp, st));
-    else
-        ACCERL_CUDA_TRY(launch_ingest_f32((const float *)obs_dev, p->s_input, x, B, p->in_c,
-                                          p->in_cp, st));
-    for (const LayerPlan &L : p->layers) {
-        const int8_t *in = p->bufs[L.in_buf].ptr;
-        int8_t *o = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
-        if (L.kind == ACCERL_CONV2D) {
-            const int8_t *skip = L.skip_buf >= 0 ? p->bufs[L.skip_buf].ptr : nullptr;
-            ACCERL_CUDA_TRY(launch_conv_generic(L, in, skip, o, B, st));
-        } else if (L.kind == ACCERL_FC) {
-            ACCERL_CUDA_TRY(launch_fc_generic(L, in, o, logits_dev, B, st));
-        } else {
-            ACCERL_CUDA_TRY(launch_maxpool_generic(L, in, o, B, st));
-        }
+    return run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev,
+                     (cudaStream_t)cuda_stream, nullptr);
+}
+
+accerl_status accerl_policy_act_timed(accerl_policy *p, const void *obs_dev,
+                                      const float *uniforms_dev, int32_t batch, float *logits_dev,
+                                      int32_t *actions_dev, float *logp_dev, void *cuda_stream,
+                                      float *launch_ms_host, int32_t launch_ms_len)
+{
+    if (!p || !launch_ms_host || launch_ms_len < (int32_t)p->steps.size()) {
+        set_error("act_timed: launch_ms_host must hold launches_per_act floats");
+        return ACCERL_ERR_INVALID_ARG;
     }
-    ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev, logp_dev,
-                                  st));
+    accerl_status v = check_act_args(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev,
+                                     logp_dev);
+    if (v != ACCERL_OK) return v;
+    DeviceGuard guard(p->device);
+    while (p->events.size() < p->steps.size() + 1) {
+        cudaEvent_t ev;
+        ACCERL_CUDA_TRY(cudaEventCreate(&ev));
+        p->events.push_back(ev);
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    v = run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev, st,
+                  p->events.data());
+    if (v != ACCERL_OK) return v;
+    ACCERL_CUDA_TRY(cudaStreamSynchronize(st));
+    for (size_t i = 0; i < p->steps.size(); ++i)
+        ACCERL_CUDA_TRY(cudaEventElapsedTime(&launch_ms_host[i], p->events[i], p->events[i + 1]));
     return ACCERL_OK;
 }
 
@@ -598,22 +681,22 @@ accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t 
     if (n_actions) *n_actions = p->n_actions;
     if (workspace_bytes) *workspace_bytes = p->workspace_bytes;
     std::string s;
-    char line[256];
+    char line[320];
     int launches = 0;
-    snprintf(line, sizeof(line), "input %dx%dx%d -> int8 NHWC via %s\n", p->in_c, p->in_h, p->in_w,
-             p->in_kind == ACCERL_IN_U8_NCHW ? "ingest_u8_kernel" : "ingest_f32_kernel");
-    s += line;
-    ++launches;
-    for (size_t i = 0; i < p->layers.size(); ++i) {
-        const LayerPlan &L = p->layers[i];
-        snprintf(line, sizeof(line), "layer %zu: %s %dx%dx%d -> %dx%dx%d via %s\n", i,
-                 L.kind == ACCERL_CONV2D ? "conv" : (L.kind == ACCERL_FC ? "fc" : "maxpool"),
-                 L.in_c, L.in_h, L.in_w, L.out_c, L.out_h, L.out_w, L.how.c_str());
+    for (const Step &t : p->steps) {
+        if (t.layer >= 0) {
+            const LayerPlan &L = p->layers[t.layer];
+            snprintf(line, sizeof(line), "launch %d: %s covers %s (%s %dx%dx%d -> %dx%dx%d)\n",
+                     launches, t.kernel.c_str(), t.covers.c_str(),
+                     L.kind == ACCERL_CONV2D ? "conv" : (L.kind == ACCERL_FC ? "fc" : "maxpool"),
+                     L.in_c, L.in_h, L.in_w, L.out_c, L.out_h, L.out_w);
+        } else {
+            snprintf(line, sizeof(line), "launch %d: %s covers %s\n", launches, t.kernel.c_str(),
+                     t.covers.c_str());
+        }
         s += line;
         ++launches;
     }
-    s += "sampling via sample_warp_kernel\n";
-    ++launches;
     if (launches_per_act) *launches_per_act = launches;
     if (plan_buf && plan_buf_bytes) {
         size_t n = std::min(plan_buf_bytes - 1, s.size());

@@ -339,11 +339,16 @@ __global__ void sample_warp_kernel(const float *__restrict__ logits, const float
     float m = z;
 #pragma unroll
     for (int o = WIDTH / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o, WIDTH));
-    float e = live ? expf(z - m) : 0.f;
+    // The first maximal lane contributes exp(0) = 1 exactly; summing only the others and
+    // taking log1p keeps log-probs near zero accurate to a few ulps of themselves.
+    const unsigned seg_mask = (WIDTH == 32 ? 0xffffffffu : ((1u << WIDTH) - 1u)) << (seg * WIDTH);
+    const unsigned ismax = __ballot_sync(0xffffffffu, live && z == m) & seg_mask;
+    const int amax = ismax ? __ffs(ismax) - 1 - seg * WIDTH : 0;
+    float e = (live && sl != amax) ? expf(z - m) : 0.f;
     float s = e;
 #pragma unroll
     for (int o = WIDTH / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o, WIDTH);
-    float lp = live ? z - m - logf(s) : 0.f;
+    float lp = live ? (z - m) - log1pf(s) : 0.f;
     float p = live ? expf(lp) : 0.f;
     float cdf = p;  // inclusive scan within the segment
 #pragma unroll
@@ -353,7 +358,6 @@ __global__ void sample_warp_kernel(const float *__restrict__ logits, const float
     }
     float uu = row < B ? u[row] : 2.f;
     unsigned hit = __ballot_sync(0xffffffffu, live && uu < cdf);
-    unsigned seg_mask = (WIDTH == 32 ? 0xffffffffu : ((1u << WIDTH) - 1u)) << (seg * WIDTH);
     unsigned h = hit & seg_mask;
     int a = h ? (__ffs(h) - 1 - seg * WIDTH) : (A - 1);
     float lpa = __shfl_sync(0xffffffffu, lp, seg * WIDTH + a);
@@ -375,16 +379,21 @@ __global__ void sample_wide_kernel(const float *__restrict__ logits, const float
     float m = -INFINITY;
     for (int i = lane; i < A; i += 32) m = fmaxf(m, z[i]);
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-    float s = 0.f;
-    for (int i = lane; i < A; i += 32) s += expf(z[i] - m);
+    int amax = A;  // first index that attains the maximum
+    for (int i = lane; i < A; i += 32)
+        if (z[i] == m) { amax = i; break; }
+    for (int o = 16; o > 0; o >>= 1) amax = min(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    float s = 0.f;  // sum over all but the maximal term, which is exp(0) = 1
+    for (int i = lane; i < A; i += 32)
+        if (i != amax) s += expf(z[i] - m);
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float lse = m + logf(s), uu = u[row];
+    const float l1p = log1pf(s), uu = u[row];
     float base = 0.f;
     int a = A - 1;
     bool found = false;
     for (int i0 = 0; i0 < A && !found; i0 += 32) {
         int i = i0 + lane;
-        float p = i < A ? expf(z[i] - lse) : 0.f, cdf = p;
+        float p = i < A ? expf((z[i] - m) - l1p) : 0.f, cdf = p;
         for (int o = 1; o < 32; o <<= 1) {
             float v = __shfl_up_sync(0xffffffffu, cdf, o);
             if (lane >= o) cdf += v;
@@ -399,7 +408,7 @@ __global__ void sample_wide_kernel(const float *__restrict__ logits, const float
     }
     if (lane == 0) {
         actions[row] = a;
-        logp[row] = z[a] - lse;
+        logp[row] = (z[a] - m) - l1p;
     }
 }
 

@@ -45,6 +45,14 @@ struct LayerPlan {
     std::string how;               // which kernel serves the layer (for accerl_policy_info)
 };
 
+// One kernel launch of the plan: which kernel, and which part of the path it covers
+// ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
+struct Step {
+    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE } kind;
+    int layer = -1;
+    std::string kernel, covers;
+};
+
 struct DeviceBuf {
     int8_t *ptr = nullptr;
     size_t bytes_per_state = 0;
@@ -61,12 +69,14 @@ struct accerl_policy {
     uint32_t flags = 0;
     int n_actions = 0;
     std::vector<accerl::LayerPlan> layers;
+    std::vector<accerl::Step> steps;      // the launch sequence of one act call
     std::vector<accerl::DeviceBuf> bufs;  // bufs[0] holds the quantised input
     int8_t *lut = nullptr;                // device, 256-entry uint8 -> int8 input table
     int *status_word = nullptr;           // device, set by kernels whose bounded waits give up
     size_t workspace_bytes = 0;
     std::vector<void *> owned;            // every device allocation, for destroy
     cudaStream_t last_stream = nullptr;
+    std::vector<cudaEvent_t> events;      // steps.size() + 1 events, created on first timed call
     // host-call staging (allocated on first accerl_policy_act_host)
     void *st_obs = nullptr;
     float *st_u = nullptr, *st_logits = nullptr, *st_logp = nullptr;
