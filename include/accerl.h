@@ -148,6 +148,43 @@ accerl_status accerl_policy_act_timed(accerl_policy *p, const void *obs_dev,
                                       float *launch_ms_host, int32_t launch_ms_len);
 
 /*
+ * The Actor step for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for deployment, not for the method.)
+ *
+ * Who needs it: an Actor that shares its GPU with a Learner or with other Actors whose framework
+ * allocators have already claimed the free HBM, a real-time control loop that cannot afford the
+ * device-wide synchronisation an allocation may imply, or any host that has been told to keep its
+ * device footprint fixed after start-up.  For such callers a workspace sized by `max_batch` at
+ * create time, or the staging buffers accerl_policy_act_host allocates on first use, are not an
+ * option.  Create the handle with max_batch = 1 (it then owns little beyond the weights) and step
+ * through this call: it computes exactly what accerl_policy_act computes, with the plain
+ * CUDA-core kernels, but keeps all int8 activations in a fixed array of
+ * ACCERL_NOALLOC_SCRATCH_BYTES bytes that is part of the library image.  Every GPU on which the
+ * library's kernels get loaded holds that array until the process exits.
+ *
+ * Same arguments, ownership and alignment rules as accerl_policy_act, except that `batch` is not
+ * limited by the handle's max_batch but by the array: a batch whose activations do not fit is
+ * rejected with ACCERL_ERR_BATCH_TOO_LARGE and a message that gives both sizes (Nature-CNN fits
+ * about 1400 states).  The call enqueues on `cuda_stream`, returns without synchronising, and calls
+ * no cudaMalloc / cudaFree or any other allocating routine.
+ *
+ * First call on a device: the library asks the CUDA runtime for the array's address on that
+ * device (once per device, remembered afterwards).  Make this first call during start-up, before
+ * any stream capture is begun.
+ *
+ * Sharing: all handles and all calls in the process use the same array, and it keeps whatever
+ * the previous call left in it.  Nothing in it has to start at zero -- every byte a kernel reads
+ * was written earlier in the same call -- so no clearing is done.  Two calls that overlap on the
+ * GPU (different streams, or different threads without ordering) race on the array and corrupt
+ * each other; order them on one stream or with events.
+ */
+#define ACCERL_NOALLOC_SCRATCH_BYTES (64u * 1024u * 1024u)
+accerl_status accerl_policy_act_noalloc(accerl_policy *p, const void *obs_dev,
+                                        const float *uniforms_dev, int32_t batch,
+                                        float *logits_dev, int32_t *actions_dev, float *logp_dev,
+                                        void *cuda_stream);
+
+/*
  * The same step for callers whose data lives in HOST memory (an Actor process that steps its
  * environments on the CPU, Section 2.1): copies obs and uniforms to device staging buffers owned
  * by the handle, runs accerl_policy_act, copies the three results back and waits for them.

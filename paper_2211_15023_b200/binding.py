@@ -51,6 +51,7 @@ def library() -> C.CDLL:
                                              C.POINTER(LayerDesc), i32, i32, C.c_uint32, i32]
         lib.accerl_policy_act.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
         lib.accerl_policy_act_timed.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, i32]
+        lib.accerl_policy_act_noalloc.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
         lib.accerl_policy_act_host.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp]
         lib.accerl_policy_read_activation.argtypes = [vp, i32, i32, vp, C.c_size_t]
         lib.accerl_policy_check.argtypes = [vp]
@@ -60,7 +61,7 @@ def library() -> C.CDLL:
         lib.accerl_policy_destroy.restype = None
         lib.accerl_last_error.restype = C.c_char_p
         lib.accerl_version.restype = C.c_char_p
-        for f in ("create", "act", "act_timed", "act_host", "read_activation", "check", "info"):
+        for f in ("create", "act", "act_timed", "act_noalloc", "act_host", "read_activation", "check", "info"):
             getattr(lib, "accerl_policy_" + f).restype = C.c_int
         _LIB = lib
     return _LIB
@@ -150,6 +151,12 @@ class Policy:
                                                  out[1].data_ptr(), out[2].data_ptr(), stream,
                                                  ms.ctypes.data, n))
         return ms
+
+    def act_noalloc_raw(self, obs_ptr, u_ptr, batch, logits_ptr, actions_ptr, logp_ptr,
+                        stream=0) -> int:
+        """accerl_policy_act_noalloc with raw device addresses; returns the status code."""
+        return library().accerl_policy_act_noalloc(self._h, obs_ptr, u_ptr, batch, logits_ptr,
+                                                   actions_ptr, logp_ptr, stream)
 
     def act_raw(self, obs_ptr, u_ptr, batch, logits_ptr, actions_ptr, logp_ptr, stream=0) -> int:
         """Unchecked pass-through returning the status code (for ABI tests)."""
