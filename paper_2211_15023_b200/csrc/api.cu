@@ -204,6 +204,18 @@ void pack_generic(const accerl_layer_desc &d, LayerPlan &L, std::vector<int32_t>
 }
 
 }  // namespace
+
+accerl_status upload_bytes(accerl_policy *p, const void *host, size_t bytes, void **dev)
+{
+    *dev = nullptr;
+    void *d = nullptr;
+    ACCERL_CUDA_TRY(cudaMalloc(&d, bytes < 16 ? 16 : bytes));
+    p->owned.push_back(d);
+    ACCERL_CUDA_TRY(cudaMemcpy(d, host, bytes, cudaMemcpyHostToDevice));
+    *dev = d;
+    return ACCERL_OK;
+}
+
 }  // namespace accerl
 
 using namespace accerl;
@@ -266,6 +278,20 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
         case Step::POOL_GENERIC:
             ACCERL_CUDA_TRY(launch_maxpool_generic(*L, in, o, B, st));
             break;
+        case Step::INGEST_S2D:
+            ACCERL_CUDA_TRY(launch_ingest_u8_s2d((const uint8_t *)obs_dev, p->lut,
+                                                 p->bufs[p->layers[0].in_buf].ptr, B, p->in_c,
+                                                 p->in_h, p->in_w, p->tensor_s2d[0], st));
+            break;
+        case Step::TC_GEMM: {
+            TcStep &t = p->tc_steps[s.tc];
+            TcGemmParams prm = t.prm;
+            prm.batch = B;
+            prm.m_tiles = (int)(((long long)B * prm.rows_per_image + 127) / 128);
+            prm.logits = prm.logits_mode ? logits_dev : nullptr;
+            ACCERL_CUDA_TRY(tc_launch(t.map_a, t.map_b, prm, t.resident_b, p->sm_count, st));
+            break;
+        }
         case Step::SAMPLE:
             ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev,
                                           logp_dev, st));
@@ -504,6 +530,25 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         ss.covers = "sample";
         p->steps.push_back(ss);
     }
+    p->tensor_s2d.assign(n_layers + 1, 1);
+    {
+        cudaDeviceProp prop;
+        cudaError_t pe = cudaGetDeviceProperties(&prop, device);
+        if (pe != cudaSuccess) {
+            set_error("create: cudaGetDeviceProperties: %s", cudaGetErrorString(pe));
+            return fail(ACCERL_ERR_CUDA);
+        }
+        p->sm_count = prop.multiProcessorCount;
+        if (prop.major != 10) {
+            set_error("create: this library is built for sm_100a only (device is sm_%d%d)",
+                      prop.major, prop.minor);
+            return fail(ACCERL_ERR_UNSUPPORTED);
+        }
+    }
+    if (!(flags & ACCERL_FLAG_FORCE_GENERIC)) {
+        bool used = false;
+        if ((st = build_tc_plan(p, layers, n_layers, &used)) != ACCERL_OK) return fail(st);
+    }
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         set_error("create: %s", cudaGetErrorString(e));
@@ -620,6 +665,7 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
         return ACCERL_ERR_INVALID_ARG;
     }
     int C, H, W, Cp, buf;
+    const int s2 = p->tensor_s2d[layer + 1];
     if (layer < 0) {
         C = p->in_c; H = p->in_h; W = p->in_w; Cp = p->in_cp; buf = p->layers[0].in_buf;
     } else {
@@ -646,7 +692,8 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
             for (int y = 0; y < H; ++y)
                 for (int x = 0; x < W; ++x)
                     dst[(((size_t)b * C + c) * H + y) * W + x] =
-                        tmp[(((size_t)b * H + y) * W + x) * Cp + c];
+                        tmp[((((size_t)b * (H / s2) + y / s2) * (W / s2) + x / s2) * s2 * s2 +
+                             (y % s2) * s2 + x % s2) * Cp + c];
     return ACCERL_OK;
 }
 

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "accerl.h"
+#include "tc_gemm.h"
 
 namespace accerl {
 
@@ -48,9 +49,19 @@ struct LayerPlan {
 // One kernel launch of the plan: which kernel, and which part of the path it covers
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
-    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE } kind;
+    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM } kind;
     int layer = -1;
+    int tc = -1;  // index into accerl_policy::tc_steps for TC_GEMM
     std::string kernel, covers;
+};
+
+// One launch of the tensor-core contraction: TMA descriptors (built once, for max_batch rows) and
+// the parameter block; batch-dependent fields are filled in per call.
+struct TcStep {
+    alignas(64) unsigned char map_a[128];
+    alignas(64) unsigned char map_b[128];
+    TcGemmParams prm;
+    bool resident_b = false;
 };
 
 struct DeviceBuf {
@@ -70,6 +81,9 @@ struct accerl_policy {
     int n_actions = 0;
     std::vector<accerl::LayerPlan> layers;
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
+    std::vector<accerl::TcStep> tc_steps;
+    std::vector<int> tensor_s2d;          // space-to-depth factor of tensor t at [t + 1]
+    int sm_count = 0;
     std::vector<accerl::DeviceBuf> bufs;  // bufs[0] holds the quantised input
     int8_t *lut = nullptr;                // device, 256-entry uint8 -> int8 input table
     int *status_word = nullptr;           // device, set by kernels whose bounded waits give up
@@ -99,5 +113,11 @@ cudaError_t launch_maxpool_generic(const LayerPlan &L, const int8_t *in, int8_t 
                                    cudaStream_t st);
 cudaError_t launch_sample(const float *logits, const float *u, int B, int A, int32_t *actions,
                           float *logp, cudaStream_t st);
+
+// tensor-core plan (tc_plan.cu): replaces p->steps when the whole network qualifies; returns
+// ACCERL_OK with *used = false when it does not
+accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
+                            bool *used);
+accerl_status upload_bytes(accerl_policy *p, const void *host, size_t bytes, void **dev);
 
 }  // namespace accerl

@@ -1,0 +1,439 @@
+// int8 tensor-core contraction for sm_100a: tcgen05.mma kind::i8 with int32 accumulators in
+// tensor memory, operands staged in shared memory by TMA, and the requant / bias / ReLU / int8
+// store epilogue fused behind it.  One kernel serves fully connected layers and convolutions.
+//
+// Convolutions run as "shifted-row" implicit GEMMs.  The activation tensor is stored so that one
+// GEMM row is one position (n, Y, X) of a stride-1 grid and every filter tap is a fixed row
+// offset: a conv with stride s and window k = s*t on an NHWC tensor is a t x t stride-1 conv on
+// its space-to-depth(s) form [H/s][W/s][s*s*C].  The K loop then walks a list of chunks, each a
+// TMA box [128 rows][chunk bytes] fetched at (row0 + row_off[j], col_off[j]); rows whose window
+// would leave the image are computed and thrown away by the epilogue.
+//
+// Roles inside a CTA (192 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
+// the MMAs, warps 2..5 drain accumulators (each its own 32-lane quarter of tensor memory),
+// requantise and store.  The kernel is persistent: CTAs stride over the tile list, smem stages
+// and accumulator stages are ring buffers guarded by mbarriers.  Every wait is bounded; a wait
+// that gives up sets the policy's status word and all roles leave.
+#include <cuda.h>
+
+#include "epilogue.cuh"
+#include "internal.h"
+#include "tc_gemm.h"
+
+#include <algorithm>
+
+namespace accerl {
+
+namespace {
+
+constexpr int kTileM = 128;
+constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait: gives up after kWaitLimitCycles or as soon as another role has given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int *status, int code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *abort_flag = 1;
+            atomicOr(status, code);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+// shared-memory matrix descriptor, K-major, swizzled rows of `chunk_bytes` (32 / 64 / 128)
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, int chunk_bytes)
+{
+    const uint64_t layout = chunk_bytes == 128 ? 2 : (chunk_bytes == 64 ? 4 : 6);
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);            // start address
+    d |= (uint64_t)1 << 16;                                 // leading byte offset (unused here)
+    d |= (uint64_t)((8 * chunk_bytes) >> 4) << 32;          // stride between 8-row groups
+    d |= (uint64_t)1 << 46;                                 // descriptor version
+    d |= layout << 61;
+    return d;
+}
+
+__device__ __forceinline__ void mma_i8(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc,
+                                       uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n}\n"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void mma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar)
+                 : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+struct __align__(8) Barriers {
+    uint64_t full[kTcMaxStages], empty[kTcMaxStages];
+    uint64_t acc_full[kTcMaxAccStages], acc_empty[kTcMaxAccStages];
+    uint64_t b_ready;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+}  // namespace
+
+template <bool RESIDENT_B>
+__global__ void __launch_bounds__(192, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const TcGemmParams p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    // the dynamic region is only guaranteed 16-byte aligned; swizzled tiles need 1024
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ Barriers bars;
+    __shared__ __align__(16) float s_ks[kTcMaxN], s_bs[kTcMaxN];
+    for (int i = threadIdx.x; i < p.n_total; i += blockDim.x) {
+        s_ks[i] = p.kscale[i];
+        s_bs[i] = p.bias[i];
+    }
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int CH = p.chunk_bytes;
+    const int a_stage_bytes = kTileM * CH;
+    const int b_tile_bytes = p.n_tile * CH;
+    const int stage_bytes = a_stage_bytes + (RESIDENT_B ? 0 : b_tile_bytes);
+    uint8_t *resident_b = smem;
+    uint8_t *stages = smem + (RESIDENT_B ? ((p.n_chunks * b_tile_bytes + 1023) & ~1023) : 0);
+    const int n_stages = p.n_stages, n_acc = p.n_acc_stages;
+    const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;  // column stride of an accumulator stage
+    volatile int *abort_flag = &bars.abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < n_stages; ++s) {
+            mbar_init(smem_u32(&bars.full[s]), 1);
+            mbar_init(smem_u32(&bars.empty[s]), 1);
+        }
+        for (int a = 0; a < n_acc; ++a) {
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+        }
+        mbar_init(smem_u32(&bars.b_ready), 1);
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars.tmem_base)), "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = bars.tmem_base;
+
+    const int total_tiles = p.m_tiles * p.n_tiles;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            if (RESIDENT_B) {
+                mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
+                for (int j = 0; j < p.n_chunks; ++j)
+                    tma_load_2d(smem_u32(resident_b + j * b_tile_bytes), &map_b, 0, j * p.n_total,
+                                smem_u32(&bars.b_ready));
+            }
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const int mt = t / p.n_tiles, nt = t % p.n_tiles;
+                const int row0 = mt * kTileM;
+                for (int j = 0; j < p.n_chunks; ++j, ++it) {
+                    const int s = it % n_stages;
+                    const uint32_t par = ((it / n_stages) & 1) ^ 1;
+                    if (!(ok = mbar_wait(smem_u32(&bars.empty[s]), par, abort_flag, p.status, 1)))
+                        break;
+                    const uint32_t full = smem_u32(&bars.full[s]);
+                    mbar_expect_tx(full, (uint32_t)stage_bytes);
+                    uint8_t *st = stages + (size_t)s * stage_bytes;
+                    tma_load_2d(smem_u32(st), &map_a, p.col_off[j], row0 + p.row_off[j], full);
+                    if (!RESIDENT_B)
+                        tma_load_2d(smem_u32(st + a_stage_bytes), &map_b, 0,
+                                    j * p.n_total + nt * p.n_tile, full);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) |
+                                   ((uint32_t)(p.n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            bool ok = true;
+            if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
+            int it = 0, tile_i = 0;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
+                const int a = tile_i % n_acc;
+                const uint32_t apar = ((tile_i / n_acc) & 1) ^ 1;
+                if (!(ok = mbar_wait(smem_u32(&bars.acc_empty[a]), apar, abort_flag, p.status, 4)))
+                    break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
+                for (int j = 0; j < p.n_chunks; ++j, ++it) {
+                    const int s = it % n_stages;
+                    const uint32_t par = (it / n_stages) & 1;
+                    if (!(ok = mbar_wait(smem_u32(&bars.full[s]), par, abort_flag, p.status, 8)))
+                        break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = smem_u32(stages + (size_t)s * stage_bytes);
+                    const uint32_t b_addr = RESIDENT_B ? smem_u32(resident_b + j * b_tile_bytes)
+                                                       : a_addr + a_stage_bytes;
+                    for (int k = 0; k < CH; k += 32)
+                        mma_i8(d_tmem, make_desc(a_addr + k, CH), make_desc(b_addr + k, CH), idesc,
+                               (j | k) != 0);
+                    mma_commit(smem_u32(&bars.empty[s]));  // frees the stage when the MMAs retire
+                }
+                if (ok) mma_commit(smem_u32(&bars.acc_full[a]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------- epilogue (warps 2..5)
+        const int q = warp & 3;  // this warp's quarter of tensor memory
+        int tile_i = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
+            const int mt = t / p.n_tiles, nt = t % p.n_tiles;
+            const int a = tile_i % n_acc;
+            const uint32_t apar = (tile_i / n_acc) & 1;
+            ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const long long m = (long long)mt * kTileM + q * 32 + lane;
+            // which output position is this GEMM row?
+            const long long n = m / p.rows_per_image;
+            const int r = (int)(m - n * p.rows_per_image);
+            const int Y = r / p.grid_w, X = r - Y * p.grid_w;
+            const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
+            const int s2 = p.out_s2d;
+            const long long out_row = n * p.out_rows_per_image + (Y / s2) * p.out_grid_w + X / s2;
+            const int col0 = nt * p.n_tile;
+            int8_t *dst = p.out + out_row * p.out_pitch + ((Y % s2) * s2 + X % s2) * p.n_total + col0;
+            float *ldst = p.logits ? p.logits + m * p.n_actions : nullptr;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_cols);
+            for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+                int acc[16];
+                tmem_ld16(taddr + c0, acc);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (c0 + 16 >= p.n_tile) {
+                    // all of this warp's reads of the stage are done: hand it back to the MMA warp
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.acc_empty[a]));
+                }
+                if (!valid) continue;
+                float ks[16], bs[16];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    const float4 kv = *reinterpret_cast<const float4 *>(&s_ks[col0 + c0 + 4 * g]);
+                    const float4 bv = *reinterpret_cast<const float4 *>(&s_bs[col0 + c0 + 4 * g]);
+                    ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                    bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+                }
+                if (ldst) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (col0 + c0 + i < p.n_actions)
+                            ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
+                } else {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint32_t word = 0;
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            const int i = 4 * g + b;
+                            float y = epilogue_float(acc[i], ks[i], bs[i], p.relu_out);
+                            word |= (uint32_t)(uint8_t)requant(y, p.s_out) << (8 * b);
+                        }
+                        w[g] = word;
+                    }
+                    *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (*abort_flag) {
+        // let copies that are still in flight land before the shared memory goes away
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) ==
+                cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)sym;
+    }
+    return fn;
+}
+
+// 2-D uint8 tensor [rows][row_bytes] with pitch `pitch`; box [box_rows][box_bytes], swizzled.
+accerl_status tc_make_map(void *map_out, const void *base, long long rows, int row_bytes,
+                          long long pitch, int box_rows, int box_bytes)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) {
+        set_error("cuTensorMapEncodeTiled is not available from this driver");
+        return ACCERL_ERR_CUDA;
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch};
+    cuuint32_t box[2] = {(cuuint32_t)box_bytes, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUtensorMapSwizzle sw = box_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                            : box_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                              : CU_TENSOR_MAP_SWIZZLE_32B;
+    CUresult r = fn((CUtensorMap *)map_out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, (void *)base, dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error("cuTensorMapEncodeTiled failed (%d) for rows=%lld row_bytes=%d pitch=%lld box=%dx%d",
+                  (int)r, rows, row_bytes, pitch, box_rows, box_bytes);
+        return ACCERL_ERR_CUDA;
+    }
+    return ACCERL_OK;
+}
+
+size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
+{
+    const int a_stage = kTileM * p.chunk_bytes, b_tile = p.n_tile * p.chunk_bytes;
+    size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
+    return 1024 + res + (size_t)p.n_stages * (a_stage + (resident_b ? 0 : b_tile));
+}
+
+// Choose ring sizes for a problem; returns false if even the smallest pipeline does not fit.
+bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
+{
+    const size_t limit = 227 * 1024 - 2048;
+    for (int s = kTcMaxStages; s >= 2; --s) {
+        p.n_stages = s;
+        if (tc_smem_bytes(p, resident_b) <= limit) {
+            const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
+            p.n_acc_stages = std::min(kTcMaxAccStages, 512 / acc_cols);
+            int cols = 32;
+            while (cols < p.n_acc_stages * acc_cols) cols *= 2;
+            p.tmem_cols = cols;
+            return true;
+        }
+    }
+    return false;
+}
+
+cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &p, bool resident_b,
+                      int sm_count, cudaStream_t st)
+{
+    const size_t smem = tc_smem_bytes(p, resident_b);
+    const int tiles = p.m_tiles * p.n_tiles;
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    cudaError_t e;
+    if (resident_b) {
+        e = cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem);
+        if (e != cudaSuccess) return e;
+        tc_gemm_kernel<true><<<grid, 192, smem, st>>>(*(const CUtensorMap *)map_a,
+                                                      *(const CUtensorMap *)map_b, p);
+    } else {
+        e = cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem);
+        if (e != cudaSuccess) return e;
+        tc_gemm_kernel<false><<<grid, 192, smem, st>>>(*(const CUtensorMap *)map_a,
+                                                       *(const CUtensorMap *)map_b, p);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace accerl

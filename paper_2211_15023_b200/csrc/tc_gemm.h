@@ -1,0 +1,50 @@
+// Parameters of the tensor-core contraction kernel (tc_gemm.cu).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "accerl.h"
+
+namespace accerl {
+
+constexpr int kTcMaxChunks = 64;
+constexpr int kTcMaxStages = 8;
+constexpr int kTcMaxAccStages = 4;
+constexpr int kTcMaxN = 512;
+
+struct TcGemmParams {
+    // K loop: chunk j is the TMA box at (row0 + row_off[j], col_off[j]) of the A tensor and rows
+    // [j * n_total, (j + 1) * n_total) of the packed weight tensor
+    int n_chunks, chunk_bytes;
+    int row_off[kTcMaxChunks], col_off[kTcMaxChunks];
+    // tiling
+    int m_tiles, n_tiles, n_tile, n_total;
+    int n_stages, n_acc_stages, tmem_cols;
+    // GEMM row -> output position: row = n * rows_per_image + Y * grid_w + X, kept when
+    // Y < out_h and X < out_w; stored at row n * out_rows_per_image + (Y/s) * out_grid_w + X/s,
+    // byte ((Y%s) * s + X%s) * n_total + channel, rows `out_pitch` bytes apart (s = out_s2d)
+    int batch, rows_per_image, grid_w, out_h, out_w;
+    int out_s2d, out_rows_per_image, out_grid_w, out_pitch;
+    // epilogue
+    const float *kscale, *bias;
+    float s_out;
+    int relu_out;
+    int8_t *out;
+    int logits_mode;  // 1: write fp32 logits [batch][n_actions] to `logits` instead of int8
+    float *logits;
+    int n_actions;
+    int *status;
+};
+
+accerl_status tc_make_map(void *map_out, const void *base, long long rows, int row_bytes,
+                          long long pitch, int box_rows, int box_bytes);
+bool tc_choose_pipeline(TcGemmParams &p, bool resident_b);
+size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b);
+cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &p, bool resident_b,
+                      int sm_count, cudaStream_t st);
+
+// uint8 NCHW frames -> int8 space-to-depth(s) rows [B * (H/s) * (W/s)][s*s*C]
+cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
+                                 int H, int W, int s, cudaStream_t st);
+
+}  // namespace accerl

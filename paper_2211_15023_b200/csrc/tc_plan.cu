@@ -1,0 +1,253 @@
+// Builds the tensor-core plan of a policy: which activation layouts the layers exchange, how the
+// weights are packed for the shifted-row implicit GEMM, the TMA descriptors and launch
+// parameters.  Also holds the input kernel that writes frames in space-to-depth form.
+#include <string.h>
+
+#include "epilogue.cuh"
+#include "internal.h"
+
+namespace accerl {
+
+// ---------------------------------------------------------------------------------------
+// uint8 NCHW frames -> int8 space-to-depth(s) rows, C = 4, s = 4: each thread turns one
+// 4-pixel run of all four channel planes into 16 output bytes ((dx, c) order).
+// ---------------------------------------------------------------------------------------
+__global__ void ingest_u8_s2d44_kernel(const uint8_t *__restrict__ obs,
+                                       const int8_t *__restrict__ lut, uint4 *__restrict__ out,
+                                       long long total, int H, int W)
+{
+    __shared__ int8_t s_lut[256];
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = lut[i];
+    __syncthreads();
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int Ws = W / 4, Hs = H / 4;
+    // idx = ((n * Hs + Y) * 4 + dy) * Ws + X
+    int X = (int)(idx % Ws);
+    long long t = idx / Ws;
+    int dy = (int)(t % 4);
+    t /= 4;
+    int Y = (int)(t % Hs);
+    long long n = t / Hs;
+    uint32_t plane[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        plane[c] = *reinterpret_cast<const uint32_t *>(
+            obs + ((n * 4 + c) * H + 4 * Y + dy) * W + 4 * X);
+    uint32_t w[4];
+#pragma unroll
+    for (int dx = 0; dx < 4; ++dx) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            word |= (uint32_t)(uint8_t)s_lut[(plane[c] >> (8 * dx)) & 0xff] << (8 * c);
+        w[dx] = word;
+    }
+    // row (n, Y, X) of 64 bytes, this thread's 16 bytes start at dy * 16
+    out[((n * Hs + Y) * Ws + X) * 4 + dy] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// any C, s: one thread per output byte
+__global__ void ingest_u8_s2d_any_kernel(const uint8_t *__restrict__ obs,
+                                         const int8_t *__restrict__ lut, int8_t *__restrict__ out,
+                                         long long total, int C, int H, int W, int s)
+{
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int Ws = W / s, Hs = H / s, Cs = s * s * C;
+    int b = (int)(idx % Cs);
+    long long r = idx / Cs;
+    int X = (int)(r % Ws);
+    r /= Ws;
+    int Y = (int)(r % Hs);
+    long long n = r / Hs;
+    int c = b % C, dx = (b / C) % s, dy = b / (C * s);
+    out[idx] = lut[obs[((n * C + c) * H + s * Y + dy) * W + s * X + dx]];
+}
+
+cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
+                                 int H, int W, int s, cudaStream_t st)
+{
+    if (C == 4 && s == 4 && W % 4 == 0) {
+        long long total = (long long)B * H * (W / 4);
+        ingest_u8_s2d44_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
+            obs, lut, (uint4 *)out, total, H, W);
+    } else {
+        long long total = (long long)B * C * H * W;
+        ingest_u8_s2d_any_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(obs, lut, out, total,
+                                                                                 C, H, W, s);
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// plan
+// ---------------------------------------------------------------------------------------
+
+namespace {
+
+bool conv_fits(const accerl_layer_desc &d)
+{
+    if (d.pad != 0 || d.kh % d.stride || d.in_h % d.stride || d.in_w % d.stride) return false;
+    const int cs = d.stride * d.stride * d.in_c;
+    if (cs != 32 && cs != 64 && cs != 128) return false;
+    const int t = d.kh / d.stride;
+    if (t * t > kTcMaxChunks) return false;
+    if (d.out_c % 16 || d.out_c > 256) return false;
+    if (d.skip_from >= 0) return false;
+    return true;
+}
+
+}  // namespace
+
+accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
+                            bool *used)
+{
+    *used = false;
+    if (p->in_kind != ACCERL_IN_U8_NCHW || layers[0].kind != ACCERL_CONV2D) return ACCERL_OK;
+    // ---- does every layer qualify?
+    for (int i = 0; i < n_layers; ++i) {
+        const accerl_layer_desc &d = layers[i];
+        const LayerPlan &L = p->layers[i];
+        const bool relu_in_noop = i > 0 && (layers[i - 1].flags & ACCERL_RELU_OUT);
+        if ((d.flags & ACCERL_RELU_IN) && !relu_in_noop) return ACCERL_OK;
+        if (d.kind == ACCERL_CONV2D) {
+            if (!conv_fits(d)) return ACCERL_OK;
+        } else if (d.kind == ACCERL_FC) {
+            const int K = L.in_h * L.in_w * L.in_cp;
+            if (L.in_cp != L.in_c || K % 16 || K < 128 || (K + 127) / 128 > kTcMaxChunks)
+                return ACCERL_OK;
+            if (d.flags & ACCERL_LOGITS) {
+                if (d.out_c > 256) return ACCERL_OK;
+            } else if (d.out_c % 16 || d.out_c > kTcMaxN || (d.out_c > 256 && d.out_c % 256)) {
+                return ACCERL_OK;
+            }
+        } else {
+            return ACCERL_OK;
+        }
+    }
+    // ---- layouts: a tensor is stored space-to-depth(s) when its reader is a conv of stride s
+    for (int i = 0; i < n_layers; ++i)
+        p->tensor_s2d[i] = layers[i].kind == ACCERL_CONV2D ? layers[i].stride : 1;
+    p->tensor_s2d[n_layers] = 1;
+
+    std::vector<Step> steps;
+    Step s0;
+    s0.kind = Step::INGEST_S2D;
+    s0.kernel = (p->in_c == 4 && p->tensor_s2d[0] == 4) ? "ingest_u8_s2d44_kernel"
+                                                        : "ingest_u8_s2d_any_kernel";
+    s0.covers = "ingest";
+    steps.push_back(s0);
+
+    for (int i = 0; i < n_layers; ++i) {
+        const accerl_layer_desc &d = layers[i];
+        const LayerPlan &L = p->layers[i];
+        TcStep ts;
+        memset(&ts.prm, 0, sizeof(ts.prm));
+        TcGemmParams &g = ts.prm;
+        const bool logits = (d.flags & ACCERL_LOGITS) != 0;
+        const int n_total = round_up(d.out_c, 16);
+        g.n_total = n_total;
+        g.n_tile = n_total > 256 ? 256 : n_total;
+        g.n_tiles = n_total / g.n_tile;
+        int rows_in_per_image, row_bytes;
+        std::vector<int8_t> packed;
+        if (d.kind == ACCERL_CONV2D) {
+            const int s = d.stride, t = d.kh / s, Hs = d.in_h / s, Ws = d.in_w / s;
+            const int CH = s * s * d.in_c;
+            g.chunk_bytes = CH;
+            g.n_chunks = t * t;
+            rows_in_per_image = Hs * Ws;
+            row_bytes = CH;
+            g.rows_per_image = Hs * Ws;
+            g.grid_w = Ws;
+            packed.assign((size_t)g.n_chunks * n_total * CH, 0);
+            for (int by = 0; by < t; ++by)
+                for (int bx = 0; bx < t; ++bx) {
+                    const int j = by * t + bx;
+                    g.row_off[j] = by * Ws + bx;
+                    g.col_off[j] = 0;
+                    for (int oc = 0; oc < d.out_c; ++oc)
+                        for (int dy = 0; dy < s; ++dy)
+                            for (int dx = 0; dx < s; ++dx)
+                                for (int c = 0; c < d.in_c; ++c)
+                                    packed[((size_t)j * n_total + oc) * CH + (dy * s + dx) * d.in_c + c] =
+                                        d.w[((oc * d.in_c + c) * d.kh + s * by + dy) * d.kw + s * bx + dx];
+                }
+        } else {
+            const int K = L.in_h * L.in_w * L.in_cp;
+            g.chunk_bytes = 128;
+            g.n_chunks = (K + 127) / 128;
+            rows_in_per_image = 1;
+            row_bytes = K;
+            g.rows_per_image = 1;
+            g.grid_w = 1;
+            packed.assign((size_t)g.n_chunks * n_total * 128, 0);
+            for (int j = 0; j < g.n_chunks; ++j) {
+                g.row_off[j] = 0;
+                g.col_off[j] = 128 * j;
+            }
+            for (int oc = 0; oc < d.out_c; ++oc)
+                for (int c = 0; c < L.in_c; ++c)
+                    for (int y = 0; y < L.in_h; ++y)
+                        for (int x = 0; x < L.in_w; ++x) {
+                            const int ki = (y * L.in_w + x) * L.in_cp + c;
+                            packed[((size_t)(ki / 128) * n_total + oc) * 128 + ki % 128] =
+                                d.w[(size_t)oc * d.in_c + (c * L.in_h + y) * L.in_w + x];
+                        }
+        }
+        g.out_h = L.out_h;
+        g.out_w = L.out_w;
+        const int so = p->tensor_s2d[i + 1];
+        g.out_s2d = so;
+        g.out_rows_per_image = (L.out_h / so) * (L.out_w / so);
+        g.out_grid_w = L.out_w / so;
+        g.out_pitch = so * so * n_total;
+        g.kscale = L.kscale;
+        g.bias = L.bias;
+        g.s_out = L.s_out;
+        g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
+        g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
+        g.logits_mode = logits ? 1 : 0;
+        g.n_actions = p->n_actions;
+        g.status = p->status_word;
+        // resident weights when the whole matrix fits beside a useful pipeline
+        ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * g.chunk_bytes <= 96 * 1024;
+        if (!tc_choose_pipeline(g, ts.resident_b)) {
+            ts.resident_b = false;
+            if (!tc_choose_pipeline(g, false)) {  // generic plan stays
+                p->tensor_s2d.assign(n_layers + 1, 1);
+                p->tc_steps.clear();
+                return ACCERL_OK;
+            }
+        }
+        void *w_dev = nullptr;
+        accerl_status st = upload_bytes(p, packed.data(), packed.size(), &w_dev);
+        if (st != ACCERL_OK) return st;
+        const long long rows = (long long)p->max_batch * rows_in_per_image;
+        st = tc_make_map(ts.map_a, p->bufs[L.in_buf].ptr, rows, row_bytes, row_bytes, 128,
+                         g.chunk_bytes);
+        if (st != ACCERL_OK) return st;
+        st = tc_make_map(ts.map_b, w_dev, (long long)g.n_chunks * n_total, g.chunk_bytes,
+                         g.chunk_bytes, g.n_tile, g.chunk_bytes);
+        if (st != ACCERL_OK) return st;
+        p->tc_steps.push_back(ts);
+        Step s;
+        s.kind = Step::TC_GEMM;
+        s.layer = i;
+        s.tc = (int)p->tc_steps.size() - 1;
+        s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
+        s.covers = "layer " + std::to_string(i);
+        steps.push_back(s);
+    }
+    Step ss;
+    ss.kind = Step::SAMPLE;
+    ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
+    ss.covers = "sample";
+    steps.push_back(ss);
+    p->steps = steps;
+    *used = true;
+    return ACCERL_OK;
+}
+
+}  // namespace accerl
