@@ -34,4 +34,48 @@ __device__ __forceinline__ int8_t requant(float y, float s_out)
     return (int8_t)clamp_round_i8(__fdiv_rn(y, s_out));
 }
 
+// Sixteen accumulators of one output position -> sixteen int8 codes in four words.
+//
+// Straight-line fast path: t = y * fl(1/s_out) differs from the IEEE quotient fl(y / s_out) by at
+// most 1.5 * 2^-23 * |t| (one rounding in the reciprocal, one in the product, half an ulp in the
+// quotient), i.e. by less than 2.4e-5 wherever the result is not clamped anyway (|t| <= 129).  So
+// whenever t is farther than kTieGuard from a half-integer, rint(t) equals rint of the quotient;
+// otherwise the element is redone with the exact divide.  Saturating conversion and saturating
+// packing implement the clamp to [-128, 127].
+constexpr float kTieGuard = 4e-5f;
+
+__device__ __forceinline__ uint32_t pack4_sat_s8(int a0, int a1, int a2, int a3)
+{
+    uint32_t hi, w;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, 0;" : "=r"(hi) : "r"(a3), "r"(a2));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(w) : "r"(a1), "r"(a0), "r"(hi));
+    return w;
+}
+
+__device__ __forceinline__ void requant16(const int (&acc)[16], const float (&ks)[16],
+                                          const float (&bs)[16], bool relu, float s_out,
+                                          float inv_s_out, uint32_t (&w)[4])
+{
+    int q[16];
+    float worst = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float y = epilogue_float(acc[i], ks[i], bs[i], relu);
+        const float t = __fmul_rn(y, inv_s_out);
+        q[i] = __float2int_rn(t);
+        worst = fmaxf(worst, fabsf(__fsub_rn(t, __int2float_rn(q[i]))));
+    }
+    if (worst > 0.5f - kTieGuard) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float y = epilogue_float(acc[i], ks[i], bs[i], relu);
+            const float t = __fmul_rn(y, inv_s_out);
+            if (fabsf(__fsub_rn(t, __int2float_rn(q[i]))) > 0.5f - kTieGuard)
+                q[i] = __float2int_rn(__fdiv_rn(y, s_out));
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < 4; ++g) w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
+}
+
 }  // namespace accerl

@@ -9,9 +9,10 @@
 // TMA box [128 rows][chunk bytes] fetched at (row0 + row_off[j], col_off[j]); rows whose window
 // would leave the image are computed and thrown away by the epilogue.
 //
-// Roles inside a CTA (192 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
-// the MMAs, warps 2..5 drain accumulators (each its own 32-lane quarter of tensor memory),
-// requantise and store.  The kernel is persistent: CTAs stride over the tile list, smem stages
+// Roles inside a CTA (320 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
+// the MMAs, warps 2..9 are two epilogue warpgroups that drain accumulators (each warp its own
+// 32-lane quarter of tensor memory), requantise and store; the warpgroups take alternate tiles,
+// or for wide tiles half of the columns each.  The kernel is persistent: CTAs stride over the tile list, smem stages
 // and accumulator stages are ring buffers guarded by mbarriers.  Every wait is bounded; a wait
 // that gives up sets the policy's status word and all roles leave.
 #include <cuda.h>
@@ -27,6 +28,7 @@ namespace accerl {
 namespace {
 
 constexpr int kTileM = 128;
+constexpr int kThreads = 320;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -143,7 +145,7 @@ struct __align__(8) Barriers {
 }  // namespace
 
 template <bool RESIDENT_B>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcGemmParams p)
 {
@@ -175,7 +177,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < n_acc; ++a) {
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
-            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+            mbar_init(smem_u32(&bars.acc_empty[a]), p.split_cols ? 8 : 4);
         }
         mbar_init(smem_u32(&bars.b_ready), 1);
         bars.abort_flag = 0;
@@ -257,11 +259,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else {
-        // ------------------------------------------------------------- epilogue (warps 2..5)
-        const int q = warp & 3;  // this warp's quarter of tensor memory
+        // ------------------------------------------------------------- epilogue (warps 2..9)
+        const int q = warp & 3;         // this warp's quarter of tensor memory
+        const int wg = (warp - 2) >> 2;  // epilogue warpgroup 0 / 1
+        const int c_begin = p.split_cols ? wg * (p.n_tile / 2) : 0;
+        const int c_end = p.split_cols ? c_begin + p.n_tile / 2 : p.n_tile;
         int tile_i = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
+            if (!p.split_cols && (tile_i & 1) != wg) continue;
             const int mt = t / p.n_tiles, nt = t % p.n_tiles;
             const int a = tile_i % n_acc;
             const uint32_t apar = (tile_i / n_acc) & 1;
@@ -269,23 +275,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const long long m = (long long)mt * kTileM + q * 32 + lane;
+            const int m = mt * kTileM + q * 32 + lane;
             // which output position is this GEMM row?
-            const long long n = m / p.rows_per_image;
-            const int r = (int)(m - n * p.rows_per_image);
+            const int n = m / p.rows_per_image;
+            const int r = m - n * p.rows_per_image;
             const int Y = r / p.grid_w, X = r - Y * p.grid_w;
             const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
             const int s2 = p.out_s2d;
-            const long long out_row = n * p.out_rows_per_image + (Y / s2) * p.out_grid_w + X / s2;
+            const long long out_row =
+                (long long)n * p.out_rows_per_image + (Y / s2) * p.out_grid_w + X / s2;
             const int col0 = nt * p.n_tile;
             int8_t *dst = p.out + out_row * p.out_pitch + ((Y % s2) * s2 + X % s2) * p.n_total + col0;
-            float *ldst = p.logits ? p.logits + m * p.n_actions : nullptr;
+            float *ldst = p.logits_mode ? p.logits + (long long)m * p.n_actions : nullptr;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_cols);
-            for (int c0 = 0; c0 < p.n_tile; c0 += 16) {
+            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 int acc[16];
                 tmem_ld16(taddr + c0, acc);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c0 + 16 >= p.n_tile) {
+                if (c0 + 16 >= c_end) {
                     // all of this warp's reads of the stage are done: hand it back to the MMA warp
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
@@ -307,17 +314,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
                 } else {
                     uint32_t w[4];
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint32_t word = 0;
-#pragma unroll
-                        for (int b = 0; b < 4; ++b) {
-                            const int i = 4 * g + b;
-                            float y = epilogue_float(acc[i], ks[i], bs[i], p.relu_out);
-                            word |= (uint32_t)(uint8_t)requant(y, p.s_out) << (8 * b);
-                        }
-                        w[g] = word;
-                    }
+                    requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
                     *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
@@ -424,13 +421,13 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
         e = cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem);
         if (e != cudaSuccess) return e;
-        tc_gemm_kernel<true><<<grid, 192, smem, st>>>(*(const CUtensorMap *)map_a,
+        tc_gemm_kernel<true><<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a,
                                                       *(const CUtensorMap *)map_b, p);
     } else {
         e = cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem);
         if (e != cudaSuccess) return e;
-        tc_gemm_kernel<false><<<grid, 192, smem, st>>>(*(const CUtensorMap *)map_a,
+        tc_gemm_kernel<false><<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a,
                                                        *(const CUtensorMap *)map_b, p);
     }
     return cudaGetLastError();

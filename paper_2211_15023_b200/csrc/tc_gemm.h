@@ -27,8 +27,9 @@ struct TcGemmParams {
     int out_s2d, out_rows_per_image, out_grid_w, out_pitch;
     // epilogue
     const float *kscale, *bias;
-    float s_out;
+    float s_out, inv_s_out;
     int relu_out;
+    int split_cols;  // 1: both epilogue warpgroups share a tile (half the columns each)
     int8_t *out;
     int logits_mode;  // 1: write fp32 logits [batch][n_actions] to `logits` instead of int8
     float *logits;

@@ -126,6 +126,9 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             return ACCERL_OK;
         }
     }
+    for (int i = 0; i < n_layers; ++i)
+        if ((long long)p->max_batch * p->layers[i].in_h * p->layers[i].in_w + 256 >= (1LL << 31))
+            return ACCERL_OK;  // GEMM row indices are 32-bit
     // ---- layouts: a tensor is stored space-to-depth(s) when its reader is a conv of stride s
     for (int i = 0; i < n_layers; ++i)
         p->tensor_s2d[i] = layers[i].kind == ACCERL_CONV2D ? layers[i].stride : 1;
@@ -206,6 +209,11 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         g.kscale = L.kscale;
         g.bias = L.bias;
         g.s_out = L.s_out;
+        {
+            volatile float inv = 1.0f / L.s_out;  // IEEE reciprocal, rounded once
+            g.inv_s_out = inv;
+        }
+        g.split_cols = g.n_tile >= 128 ? 1 : 0;
         g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
         g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
         g.logits_mode = logits ? 1 : 0;

@@ -145,6 +145,44 @@ def test_odd_shapes_padding_stride_pool_residual():
     g.close()
 
 
+def test_exact_ties_on_the_tensor_core_path():
+    """Power-of-two scales make many epilogue quotients land exactly on k + 0.5: the requantiser
+    must round them to even exactly as the IEEE divide + rintf of the definition does."""
+    import paper_2211_15023_b200 as P
+    from oracle import net as ON
+    name = "student_cnn_b8192"
+    pol = W.drawn_int8_policy(name, seed=123)
+    b = 24
+    obs, u = W.observations(name, b, seed=9), W.uniforms(name, b, seed=10)
+    pol["s_input"] = np.float32(2.0 ** -7)
+    x = ON.ingest("u8", obs, pol["s_input"]).reshape((b,) + pol["in_shape"])
+    s_prev, ties = pol["s_input"], 0
+    for l in pol["layers"]:
+        l["s_in"] = s_prev
+        l["s_w"] = np.full(l["out_c"], 2.0 ** -7, np.float32)
+        if l["kind"] == "fc":
+            x = x.reshape(b, -1, 1, 1)
+        acc = ON.layer_acc(l, x)
+        y0 = ON.layer_float(dict(l, bias=np.zeros(l["out_c"], np.float32)), acc)
+        if l["logits"]:
+            break
+        e = int(np.ceil(np.log2(np.abs(y0).max() / 127.0))) - 1      # some saturation on purpose
+        l["s_out"] = np.float32(2.0 ** e)
+        l["bias"] = (np.round(l["bias"] / (l["s_out"] / 2)) * (l["s_out"] / 2)).astype(np.float32)
+        y = ON.layer_float(l, acc)
+        frac = np.abs(y / l["s_out"]) % 1.0
+        ties += int(((frac == 0.5) & (np.abs(y / l["s_out"]) < 127)).sum())
+        x = ON.requant(y, l["s_out"])
+        s_prev = l["s_out"]
+    assert ties > 200, ties
+    ref = oracle.forward(pol, obs, u)
+    g = P.Policy(pol, b, flags=1)
+    assert "tc_gemm" in g.info()["plan"]
+    out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+    compare(ref, *out, taps=g.read_activation)
+    g.close()
+
+
 def test_abi_rejects_bad_calls_without_launching():
     import paper_2211_15023_b200 as P
     pol = calibrated("cartpole_mlp")
