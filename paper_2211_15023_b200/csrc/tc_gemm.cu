@@ -9,10 +9,11 @@
 // TMA box [128 rows][chunk bytes] fetched at (row0 + row_off[j], col_off[j]); rows whose window
 // would leave the image are computed and thrown away by the epilogue.
 //
-// Roles inside a CTA (320 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
-// the MMAs, warps 2..9 are two epilogue warpgroups that drain accumulators (each warp its own
-// 32-lane quarter of tensor memory), requantise and store; the warpgroups take alternate tiles,
-// or for wide tiles half of the columns each.  The kernel is persistent: CTAs stride over the tile list, smem stages
+// Roles inside a CTA (576 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
+// the MMAs, warps 2..17 are four epilogue warpgroups that drain accumulators (each warp its own
+// 32-lane quarter of tensor memory), requantise and store; the warpgroups take tiles in turn,
+// or for wide tiles a quarter of the columns each.  The epilogue is latency bound per warp, so
+// four warps per scheduler are what keeps the issue slots busy.  The kernel is persistent: CTAs stride over the tile list, smem stages
 // and accumulator stages are ring buffers guarded by mbarriers.  Every wait is bounded; a wait
 // that gives up sets the policy's status word and all roles leave.
 #include <cuda.h>
@@ -28,7 +29,8 @@ namespace accerl {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kThreads = 320;
+constexpr int kEpiGroups = 4;                       // epilogue warpgroups
+constexpr int kThreads = 64 + 128 * kEpiGroups;     // producer warp + MMA warp + epilogue
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -134,6 +136,21 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&r)[16])
         : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, int (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]),
+          "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+
 struct __align__(8) Barriers {
     uint64_t full[kTcMaxStages], empty[kTcMaxStages];
     uint64_t acc_full[kTcMaxAccStages], acc_empty[kTcMaxAccStages];
@@ -161,9 +178,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int CH = p.chunk_bytes;
-    const int a_stage_bytes = kTileM * CH;
+    const int a_chunk_bytes = kTileM * CH;
     const int b_tile_bytes = p.n_tile * CH;
-    const int stage_bytes = a_stage_bytes + (RESIDENT_B ? 0 : b_tile_bytes);
+    const int stage_bytes = p.group * (a_chunk_bytes + (RESIDENT_B ? 0 : b_tile_bytes));
     uint8_t *resident_b = smem;
     uint8_t *stages = smem + (RESIDENT_B ? ((p.n_chunks * b_tile_bytes + 1023) & ~1023) : 0);
     const int n_stages = p.n_stages, n_acc = p.n_acc_stages;
@@ -177,7 +194,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < n_acc; ++a) {
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
-            mbar_init(smem_u32(&bars.acc_empty[a]), p.split_cols ? 8 : 4);
+            mbar_init(smem_u32(&bars.acc_empty[a]), p.split_cols ? 4 * kEpiGroups : 4);
         }
         mbar_init(smem_u32(&bars.b_ready), 1);
         bars.abort_flag = 0;
@@ -197,32 +214,44 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int total_tiles = p.m_tiles * p.n_tiles;
 
+    // A smem stage holds `group` consecutive K chunks: [A chunk 0..G-1][B chunk 0..G-1].  The two
+    // single-thread issue loops below are latency bound per instruction, so they keep running
+    // stage / phase counters instead of dividing, and take one barrier round trip per stage.
+    const int G = p.group, n_groups = p.n_chunks / G;
+    const uint32_t stages_addr = smem_u32(stages), resident_addr = smem_u32(resident_b);
+    const uint32_t full0 = smem_u32(&bars.full[0]), empty0 = smem_u32(&bars.empty[0]);
+
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
         if (lane == 0) {
             if (RESIDENT_B) {
                 mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
                 for (int j = 0; j < p.n_chunks; ++j)
-                    tma_load_2d(smem_u32(resident_b + j * b_tile_bytes), &map_b, 0, j * p.n_total,
+                    tma_load_2d(resident_addr + j * b_tile_bytes, &map_b, 0, j * p.n_total,
                                 smem_u32(&bars.b_ready));
             }
-            int it = 0;
+            int s = 0;
+            uint32_t par = 1;
             bool ok = true;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int mt = t / p.n_tiles, nt = t % p.n_tiles;
-                const int row0 = mt * kTileM;
-                for (int j = 0; j < p.n_chunks; ++j, ++it) {
-                    const int s = it % n_stages;
-                    const uint32_t par = ((it / n_stages) & 1) ^ 1;
-                    if (!(ok = mbar_wait(smem_u32(&bars.empty[s]), par, abort_flag, p.status, 1)))
-                        break;
-                    const uint32_t full = smem_u32(&bars.full[s]);
+                const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
+                const int row0 = mt * kTileM, brow0 = nt * p.n_tile;
+                for (int gi = 0, j = 0; gi < n_groups; ++gi) {
+                    if (!(ok = mbar_wait(empty0 + 8 * s, par, abort_flag, p.status, 1))) break;
+                    const uint32_t full = full0 + 8 * s;
                     mbar_expect_tx(full, (uint32_t)stage_bytes);
-                    uint8_t *st = stages + (size_t)s * stage_bytes;
-                    tma_load_2d(smem_u32(st), &map_a, p.col_off[j], row0 + p.row_off[j], full);
-                    if (!RESIDENT_B)
-                        tma_load_2d(smem_u32(st + a_stage_bytes), &map_b, 0,
-                                    j * p.n_total + nt * p.n_tile, full);
+                    const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
+                    for (int c = 0; c < G; ++c, ++j) {
+                        tma_load_2d(st + c * a_chunk_bytes, &map_a, p.col_off[j], row0 + p.row_off[j],
+                                    full);
+                        if (!RESIDENT_B)
+                            tma_load_2d(st + G * a_chunk_bytes + c * b_tile_bytes, &map_b, 0,
+                                        j * p.n_total + brow0, full);
+                    }
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
                 }
             }
         }
@@ -231,43 +260,61 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) |
                                    ((uint32_t)(p.n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+            // descriptor = constant upper word | (address >> 4) in the lower word
+            const uint64_t desc_hi =
+                (uint64_t)(((uint32_t)(8 * CH) >> 4) | (1u << 14) |
+                           ((CH == 128 ? 2u : (CH == 64 ? 4u : 6u)) << 29)) << 32;
+            const uint32_t desc_lo_flags = 1u << 16;
+            const int k_steps = CH / 32;
             bool ok = true;
             if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
-            int it = 0, tile_i = 0;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
-                const int a = tile_i % n_acc;
-                const uint32_t apar = ((tile_i / n_acc) & 1) ^ 1;
+            int s = 0, a = 0;
+            uint32_t par = 0, apar = 1;
+            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
                 if (!(ok = mbar_wait(smem_u32(&bars.acc_empty[a]), apar, abort_flag, p.status, 4)))
                     break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
-                for (int j = 0; j < p.n_chunks; ++j, ++it) {
-                    const int s = it % n_stages;
-                    const uint32_t par = (it / n_stages) & 1;
-                    if (!(ok = mbar_wait(smem_u32(&bars.full[s]), par, abort_flag, p.status, 8)))
-                        break;
+                uint32_t accumulate = 0;
+                for (int gi = 0, j = 0; gi < n_groups; ++gi) {
+                    if (!(ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8))) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_addr = smem_u32(stages + (size_t)s * stage_bytes);
-                    const uint32_t b_addr = RESIDENT_B ? smem_u32(resident_b + j * b_tile_bytes)
-                                                       : a_addr + a_stage_bytes;
-                    for (int k = 0; k < CH; k += 32)
-                        mma_i8(d_tmem, make_desc(a_addr + k, CH), make_desc(b_addr + k, CH), idesc,
-                               (j | k) != 0);
-                    mma_commit(smem_u32(&bars.empty[s]));  // frees the stage when the MMAs retire
+                    const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
+                    for (int c = 0; c < G; ++c, ++j) {
+                        const uint32_t a_lo = ((st + c * a_chunk_bytes) >> 4) | desc_lo_flags;
+                        const uint32_t b_addr = RESIDENT_B ? resident_addr + j * b_tile_bytes
+                                                           : st + G * a_chunk_bytes + c * b_tile_bytes;
+                        const uint32_t b_lo = (b_addr >> 4) | desc_lo_flags;
+                        for (int k = 0; k < k_steps; ++k) {
+                            mma_i8(d_tmem, desc_hi | (a_lo + 2 * k), desc_hi | (b_lo + 2 * k), idesc,
+                                   accumulate);
+                            accumulate = 1;
+                        }
+                    }
+                    mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
+                    if (++s == n_stages) {
+                        s = 0;
+                        par ^= 1;
+                    }
                 }
                 if (ok) mma_commit(smem_u32(&bars.acc_full[a]));
+                if (++a == n_acc) {
+                    a = 0;
+                    apar ^= 1;
+                }
             }
         }
     } else {
-        // ------------------------------------------------------------- epilogue (warps 2..9)
+        // ------------------------------------------------------------- epilogue (warps 2..17)
         const int q = warp & 3;         // this warp's quarter of tensor memory
-        const int wg = (warp - 2) >> 2;  // epilogue warpgroup 0 / 1
-        const int c_begin = p.split_cols ? wg * (p.n_tile / 2) : 0;
-        const int c_end = p.split_cols ? c_begin + p.n_tile / 2 : p.n_tile;
+        const int wg = (warp - 2) >> 2;  // epilogue warpgroup
+        const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
+        const int c_begin = p.split_cols ? wg * c_span : 0;
+        const int c_end = c_begin + c_span;
         int tile_i = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
-            if (!p.split_cols && (tile_i & 1) != wg) continue;
+            if (!p.split_cols && (tile_i % kEpiGroups) != wg) continue;
             const int mt = t / p.n_tiles, nt = t % p.n_tiles;
             const int a = tile_i % n_acc;
             const uint32_t apar = (tile_i / n_acc) & 1;
@@ -288,34 +335,50 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int8_t *dst = p.out + out_row * p.out_pitch + ((Y % s2) * s2 + X % s2) * p.n_total + col0;
             float *ldst = p.logits_mode ? p.logits + (long long)m * p.n_actions : nullptr;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_cols);
-            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
-                int acc[16];
-                tmem_ld16(taddr + c0, acc);
+            for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+                const bool two = c0 + 32 <= c_end;  // 32 columns per round, 16 for a narrow tail
+                int acc[32];
+                if (two) {
+                    tmem_ld32(taddr + c0, acc);
+                } else {
+                    int lo[16];
+                    tmem_ld16(taddr + c0, lo);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) acc[i] = lo[i];
+                }
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c0 + 16 >= c_end) {
+                if (c0 + 32 >= c_end) {
                     // all of this warp's reads of the stage are done: hand it back to the MMA warp
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars.acc_empty[a]));
                 }
                 if (!valid) continue;
-                float ks[16], bs[16];
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const float4 kv = *reinterpret_cast<const float4 *>(&s_ks[col0 + c0 + 4 * g]);
-                    const float4 bv = *reinterpret_cast<const float4 *>(&s_bs[col0 + c0 + 4 * g]);
-                    ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
-                    bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
-                }
-                if (ldst) {
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1 && !two) break;
+                    const int cc = c0 + 16 * h;
+                    int part[16];
+                    float ks[16], bs[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (col0 + c0 + i < p.n_actions)
-                            ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
-                } else {
-                    uint32_t w[4];
-                    requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
-                    *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                    for (int i = 0; i < 16; ++i) part[i] = acc[16 * h + i];
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const float4 kv = *reinterpret_cast<const float4 *>(&s_ks[col0 + cc + 4 * g]);
+                        const float4 bv = *reinterpret_cast<const float4 *>(&s_bs[col0 + cc + 4 * g]);
+                        ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                        bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+                    }
+                    if (ldst) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (col0 + cc + i < p.n_actions)
+                                ldst[col0 + cc + i] = epilogue_float(part[i], ks[i], bs[i], false);
+                    } else {
+                        uint32_t w[4];
+                        requant16(part, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
+                        *reinterpret_cast<uint4 *>(dst + cc) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
                 }
             }
         }
@@ -387,15 +450,20 @@ accerl_status tc_make_map(void *map_out, const void *base, long long rows, int r
 
 size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
 {
-    const int a_stage = kTileM * p.chunk_bytes, b_tile = p.n_tile * p.chunk_bytes;
+    const int a_chunk = kTileM * p.chunk_bytes, b_tile = p.n_tile * p.chunk_bytes;
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
-    return 1024 + res + (size_t)p.n_stages * (a_stage + (resident_b ? 0 : b_tile));
+    return 1024 + res + (size_t)p.n_stages * p.group * (a_chunk + (resident_b ? 0 : b_tile));
 }
 
 // Choose ring sizes for a problem; returns false if even the smallest pipeline does not fit.
 bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
 {
-    const size_t limit = 227 * 1024 - 2048;
+    const size_t limit = 216 * 1024;  // leaves room for the static shared variables
+    // chunks per stage: the largest divisor of n_chunks that keeps a stage at or under 32 KB
+    const int per_chunk = kTileM * p.chunk_bytes + (resident_b ? 0 : p.n_tile * p.chunk_bytes);
+    p.group = 1;
+    for (int g = 1; g <= p.n_chunks; ++g)
+        if (p.n_chunks % g == 0 && g * per_chunk <= 32 * 1024) p.group = g;
     for (int s = kTcMaxStages; s >= 2; --s) {
         p.n_stages = s;
         if (tc_smem_bytes(p, resident_b) <= limit) {

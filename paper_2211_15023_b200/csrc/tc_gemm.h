@@ -20,6 +20,7 @@ struct TcGemmParams {
     // tiling
     int m_tiles, n_tiles, n_tile, n_total;
     int n_stages, n_acc_stages, tmem_cols;
+    int group;  // K chunks per shared-memory stage
     // GEMM row -> output position: row = n * rows_per_image + Y * grid_w + X, kept when
     // Y < out_h and X < out_w; stored at row n * out_rows_per_image + (Y/s) * out_grid_w + X/s,
     // byte ((Y%s) * s + X%s) * n_total + channel, rows `out_pitch` bytes apart (s = out_s2d)

@@ -213,7 +213,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             volatile float inv = 1.0f / L.s_out;  // IEEE reciprocal, rounded once
             g.inv_s_out = inv;
         }
-        g.split_cols = g.n_tile >= 128 ? 1 : 0;
+        g.split_cols = g.n_tile >= 128 ? 1 : 0;  // 128 / 256 columns: 32 / 64 per warpgroup
         g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
         g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
         g.logits_mode = logits ? 1 : 0;
