@@ -504,7 +504,7 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         if ((st = upload(p, lut, &p->lut)) != ACCERL_OK) return fail(st);
     }
     {
-        std::vector<int> zero(4, 0);
+        std::vector<int> zero(256, 0);  // word 0 is the status; the rest is trace space
         if ((st = upload(p, zero, &p->status_word)) != ACCERL_OK) return fail(st);
     }
     // ---- launch plan
@@ -752,5 +752,16 @@ accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t 
     }
     return ACCERL_OK;
 }
+
+#ifdef ACCERL_TC_TRACE
+// traced builds only: copy out and clear the per-launch role stopwatches (8 counters per launch)
+accerl_status accerl_debug_read_trace(accerl_policy *p, unsigned long long *out, int n)
+{
+    cudaDeviceSynchronize();
+    cudaMemcpy(out, p->status_word + 16, n * 8, cudaMemcpyDeviceToHost);
+    cudaMemset(p->status_word + 16, 0, n * 8);
+    return ACCERL_OK;
+}
+#endif
 
 }  // extern "C"

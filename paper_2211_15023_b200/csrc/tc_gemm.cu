@@ -38,6 +38,19 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p)
     return (uint32_t)__cvta_generic_to_shared(p);
 }
 
+// one lane of a converged warp; keeps the surrounding loop warp-uniform so that the operands of
+// the TMA / MMA instructions can live in uniform registers
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "elect.sync _|p, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -151,6 +164,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int (&r)[32])
         : "memory");
 }
 
+// Optional per-role stopwatch (build with -DACCERL_TC_TRACE): cycles spent waiting on each barrier
+// kind, summed per CTA into the words after the status word.
+#ifdef ACCERL_TC_TRACE
+#define TRACE_T0() const long long trace_t0_ = clock64()
+#define TRACE_ADD(slot) atomicAdd((unsigned long long *)(p.status + 16) + p.trace_slot * 8 + (slot), (unsigned long long)(clock64() - trace_t0_))
+#else
+#define TRACE_T0()
+#define TRACE_ADD(slot)
+#endif
+
 struct __align__(8) Barriers {
     uint64_t full[kTcMaxStages], empty[kTcMaxStages];
     uint64_t acc_full[kTcMaxAccStages], acc_empty[kTcMaxAccStages];
@@ -213,6 +236,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tmem_base = bars.tmem_base;
 
     const int total_tiles = p.m_tiles * p.n_tiles;
+#ifdef ACCERL_TC_TRACE
+    const long long trace_start = clock64();
+#endif
 
     // A smem stage holds `group` consecutive K chunks: [A chunk 0..G-1][B chunk 0..G-1].  The two
     // single-thread issue loops below are latency bound per instruction, so they keep running
@@ -223,13 +249,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            if (RESIDENT_B) {
+        {
+            if (RESIDENT_B && elect_one()) {
                 mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
                 for (int j = 0; j < p.n_chunks; ++j)
                     tma_load_2d(resident_addr + j * b_tile_bytes, &map_b, 0, j * p.n_total,
                                 smem_u32(&bars.b_ready));
             }
+            __syncwarp();
             int s = 0;
             uint32_t par = 1;
             bool ok = true;
@@ -237,17 +264,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
                 const int row0 = mt * kTileM, brow0 = nt * p.n_tile;
                 for (int gi = 0, j = 0; gi < n_groups; ++gi) {
-                    if (!(ok = mbar_wait(empty0 + 8 * s, par, abort_flag, p.status, 1))) break;
-                    const uint32_t full = full0 + 8 * s;
-                    mbar_expect_tx(full, (uint32_t)stage_bytes);
-                    const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
-                    for (int c = 0; c < G; ++c, ++j) {
-                        tma_load_2d(st + c * a_chunk_bytes, &map_a, p.col_off[j], row0 + p.row_off[j],
-                                    full);
-                        if (!RESIDENT_B)
-                            tma_load_2d(st + G * a_chunk_bytes + c * b_tile_bytes, &map_b, 0,
-                                        j * p.n_total + brow0, full);
+                    {
+                        TRACE_T0();
+                        ok = mbar_wait(empty0 + 8 * s, par, abort_flag, p.status, 1);
+                        TRACE_ADD(0);
                     }
+                    if (!ok) break;
+                    const uint32_t full = full0 + 8 * s;
+                    const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
+                    if (elect_one()) {
+                        mbar_expect_tx(full, (uint32_t)stage_bytes);
+                        for (int c = 0; c < G; ++c) {
+                            tma_load_2d(st + c * a_chunk_bytes, &map_a, p.col_off[j + c],
+                                        row0 + p.row_off[j + c], full);
+                            if (!RESIDENT_B)
+                                tma_load_2d(st + G * a_chunk_bytes + c * b_tile_bytes, &map_b, 0,
+                                            (j + c) * p.n_total + brow0, full);
+                        }
+                    }
+                    __syncwarp();
+                    j += G;
                     if (++s == n_stages) {
                         s = 0;
                         par ^= 1;
@@ -257,7 +293,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
+        {
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) |
                                    ((uint32_t)(p.n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
             // descriptor = constant upper word | (address >> 4) in the lower word
@@ -271,33 +307,48 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int s = 0, a = 0;
             uint32_t par = 0, apar = 1;
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                if (!(ok = mbar_wait(smem_u32(&bars.acc_empty[a]), apar, abort_flag, p.status, 4)))
-                    break;
+                {
+                    TRACE_T0();
+                    ok = mbar_wait(smem_u32(&bars.acc_empty[a]), apar, abort_flag, p.status, 4);
+                    TRACE_ADD(1);
+                }
+                if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
                 uint32_t accumulate = 0;
                 for (int gi = 0, j = 0; gi < n_groups; ++gi) {
-                    if (!(ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8))) break;
+                    {
+                        TRACE_T0();
+                        ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8);
+                        TRACE_ADD(2);
+                    }
+                    if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
-                    for (int c = 0; c < G; ++c, ++j) {
-                        const uint32_t a_lo = ((st + c * a_chunk_bytes) >> 4) | desc_lo_flags;
-                        const uint32_t b_addr = RESIDENT_B ? resident_addr + j * b_tile_bytes
-                                                           : st + G * a_chunk_bytes + c * b_tile_bytes;
-                        const uint32_t b_lo = (b_addr >> 4) | desc_lo_flags;
-                        for (int k = 0; k < k_steps; ++k) {
-                            mma_i8(d_tmem, desc_hi | (a_lo + 2 * k), desc_hi | (b_lo + 2 * k), idesc,
-                                   accumulate);
-                            accumulate = 1;
+                    if (elect_one()) {
+                        for (int c = 0; c < G; ++c) {
+                            const uint32_t a_lo = ((st + c * a_chunk_bytes) >> 4) | desc_lo_flags;
+                            const uint32_t b_addr = RESIDENT_B
+                                                        ? resident_addr + (j + c) * b_tile_bytes
+                                                        : st + G * a_chunk_bytes + c * b_tile_bytes;
+                            const uint32_t b_lo = (b_addr >> 4) | desc_lo_flags;
+                            for (int k = 0; k < k_steps; ++k) {
+                                mma_i8(d_tmem, desc_hi | (a_lo + 2 * k), desc_hi | (b_lo + 2 * k),
+                                       idesc, accumulate | c | k);
+                            }
                         }
+                        mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
                     }
-                    mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
+                    __syncwarp();
+                    accumulate = 1;
+                    j += G;
                     if (++s == n_stages) {
                         s = 0;
                         par ^= 1;
                     }
                 }
-                if (ok) mma_commit(smem_u32(&bars.acc_full[a]));
+                if (ok && elect_one()) mma_commit(smem_u32(&bars.acc_full[a]));
+                __syncwarp();
                 if (++a == n_acc) {
                     a = 0;
                     apar ^= 1;
@@ -318,7 +369,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int mt = t / p.n_tiles, nt = t % p.n_tiles;
             const int a = tile_i % n_acc;
             const uint32_t apar = (tile_i / n_acc) & 1;
-            ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
+            {
+                TRACE_T0();
+                ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
+                if (threadIdx.x == 64) TRACE_ADD(3);
+            }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -384,6 +439,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     }
 
+#ifdef ACCERL_TC_TRACE
+    if (lane == 0 && (warp == 0 || warp == 1 || warp == 2))
+        atomicAdd((unsigned long long *)(p.status + 16) + p.trace_slot * 8 + 4 + warp,
+                  (unsigned long long)(clock64() - trace_start));
+#endif
     // ---------------------------------------------------------------- teardown
     if (*abort_flag) {
         // let copies that are still in flight land before the shared memory goes away

@@ -36,6 +36,7 @@ struct TcGemmParams {
     float *logits;
     int n_actions;
     int *status;
+    int trace_slot;  // which block of trace counters a traced build adds to
 };
 
 accerl_status tc_make_map(void *map_out, const void *base, long long rows, int row_bytes,

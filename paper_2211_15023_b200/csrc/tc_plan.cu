@@ -219,6 +219,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         g.logits_mode = logits ? 1 : 0;
         g.n_actions = p->n_actions;
         g.status = p->status_word;
+        g.trace_slot = (int)p->tc_steps.size();
         // resident weights when the whole matrix fits beside a useful pipeline
         ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * g.chunk_bytes <= 96 * 1024;
         if (!tc_choose_pipeline(g, ts.resident_b)) {
