@@ -9,8 +9,8 @@
 // TMA box [128 rows][chunk bytes] fetched at (row0 + row_off[j], col_off[j]); rows whose window
 // would leave the image are computed and thrown away by the epilogue.
 //
-// Roles inside a CTA (576 threads): warp 0 issues TMA loads, warp 1 owns tensor memory and issues
-// the MMAs, warps 2..17 are four epilogue warpgroups that drain accumulators (each warp its own
+// Roles inside a CTA (672 threads): warp 0 issues TMA loads, warps 1..4 issue the MMAs (warp 1
+// owns the tensor-memory allocation), warps 5..20 are four epilogue warpgroups that drain accumulators (each warp its own
 // 32-lane quarter of tensor memory), requantise and store; the warpgroups take tiles in turn,
 // or for wide tiles a quarter of the columns each.  The epilogue is latency bound per warp, so
 // four warps per scheduler are what keeps the issue slots busy.  The kernel is persistent: CTAs stride over the tile list, smem stages
@@ -30,7 +30,8 @@ namespace {
 
 constexpr int kTileM = 128;
 constexpr int kEpiGroups = 4;                       // epilogue warpgroups
-constexpr int kThreads = 64 + 128 * kEpiGroups;     // producer warp + MMA warp + epilogue
+constexpr int kMmaWarps = 4;                        // MMA-issuing warps
+constexpr int kThreads = 32 * (1 + kMmaWarps) + 128 * kEpiGroups;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -203,7 +204,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int CH = p.chunk_bytes;
     const int a_chunk_bytes = kTileM * CH;
     const int b_tile_bytes = p.n_tile * CH;
-    const int stage_bytes = p.group * (a_chunk_bytes + (RESIDENT_B ? 0 : b_tile_bytes));
+    // shifted mode: a stage is one box of a_rows rows that all taps of the tile read at row offsets
+    const int stage_bytes = p.shifted ? ((p.a_rows * CH + 1023) & ~1023)
+                                      : p.group * (a_chunk_bytes + (RESIDENT_B ? 0 : b_tile_bytes));
     uint8_t *resident_b = smem;
     uint8_t *stages = smem + (RESIDENT_B ? ((p.n_chunks * b_tile_bytes + 1023) & ~1023) : 0);
     const int n_stages = p.n_stages, n_acc = p.n_acc_stages;
@@ -240,125 +243,129 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const long long trace_start = clock64();
 #endif
 
-    // A smem stage holds `group` consecutive K chunks: [A chunk 0..G-1][B chunk 0..G-1].  The two
-    // single-thread issue loops below are latency bound per instruction, so they keep running
-    // stage / phase counters instead of dividing, and take one barrier round trip per stage.
-    const int G = p.group, n_groups = p.n_chunks / G;
+    // A smem stage holds `group` consecutive K chunks: [A chunk 0..G-1][B chunk 0..G-1]; the stages
+    // of tile i (the CTA's i-th tile) are ring slots i * n_groups .. + n_groups - 1.
+    //
+    // One thread can only issue a tcgen05.mma every 150..200 cycles, far longer than the tensor
+    // pipe needs for the narrow tiles of these layers (measured: two issuing warps double the
+    // rate, an N = 64 MMA occupies the pipe for under 50 cycles).  So kMmaWarps warps issue, each
+    // for every kMmaWarps-th tile, into their own accumulator stages.
+    const int G = p.shifted ? p.n_chunks : p.group, n_groups = p.n_chunks / G;
+    const int n_mma = p.n_mma;            // issuing warps in use (never more than accumulators)
+    const int ring = n_stages / n_mma;    // ring slots per issuing warp
     const uint32_t stages_addr = smem_u32(stages), resident_addr = smem_u32(resident_b);
     const uint32_t full0 = smem_u32(&bars.full[0]), empty0 = smem_u32(&bars.empty[0]);
+    const uint32_t acc_full0 = smem_u32(&bars.acc_full[0]), acc_empty0 = smem_u32(&bars.acc_empty[0]);
+    const int my_tiles = blockIdx.x < total_tiles
+                             ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
-        {
-            if (RESIDENT_B && elect_one()) {
-                mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
-                for (int j = 0; j < p.n_chunks; ++j)
-                    tma_load_2d(resident_addr + j * b_tile_bytes, &map_b, 0, j * p.n_total,
-                                smem_u32(&bars.b_ready));
-            }
-            __syncwarp();
-            int s = 0;
-            uint32_t par = 1;
-            bool ok = true;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
-                const int row0 = mt * kTileM, brow0 = nt * p.n_tile;
-                for (int gi = 0, j = 0; gi < n_groups; ++gi) {
-                    {
-                        TRACE_T0();
-                        ok = mbar_wait(empty0 + 8 * s, par, abort_flag, p.status, 1);
-                        TRACE_ADD(0);
-                    }
-                    if (!ok) break;
-                    const uint32_t full = full0 + 8 * s;
-                    const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
-                    if (elect_one()) {
-                        mbar_expect_tx(full, (uint32_t)stage_bytes);
-                        for (int c = 0; c < G; ++c) {
-                            tma_load_2d(st + c * a_chunk_bytes, &map_a, p.col_off[j + c],
-                                        row0 + p.row_off[j + c], full);
-                            if (!RESIDENT_B)
-                                tma_load_2d(st + G * a_chunk_bytes + c * b_tile_bytes, &map_b, 0,
-                                            (j + c) * p.n_total + brow0, full);
-                        }
-                    }
-                    __syncwarp();
-                    j += G;
-                    if (++s == n_stages) {
-                        s = 0;
-                        par ^= 1;
-                    }
-                }
-            }
+        if (RESIDENT_B && elect_one()) {
+            mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
+            for (int j = 0; j < p.n_chunks; ++j)
+                tma_load_2d(resident_addr + j * b_tile_bytes, &map_b, 0, j * p.n_total,
+                            smem_u32(&bars.b_ready));
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------- MMA issuer
-        {
-            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) |
-                                   ((uint32_t)(p.n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-            // descriptor = constant upper word | (address >> 4) in the lower word
-            const uint64_t desc_hi =
-                (uint64_t)(((uint32_t)(8 * CH) >> 4) | (1u << 14) |
-                           ((CH == 128 ? 2u : (CH == 64 ? 4u : 6u)) << 29)) << 32;
-            const uint32_t desc_lo_flags = 1u << 16;
-            const int k_steps = CH / 32;
-            bool ok = true;
-            if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
-            int s = 0, a = 0;
-            uint32_t par = 0, apar = 1;
-            for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        __syncwarp();
+        bool ok = true;
+        for (int i = 0; i < my_tiles && ok; ++i) {
+            const int t = blockIdx.x + i * gridDim.x;
+            const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
+            const int row0 = mt * kTileM, brow0 = nt * p.n_tile;
+            for (int gi = 0; gi < n_groups; ++gi) {
+                const int j = gi * G;
+                // issuing warp i % n_mma owns every n_mma-th ring slot; within its slots this
+                // tile's group gi is local slot (i / n_mma) * n_groups + gi
+                const int lslot = (i / n_mma) * n_groups + gi;
+                const int s = (i % n_mma) + n_mma * (lslot % ring);
+                const uint32_t par = ((lslot / ring) & 1) ^ 1;
                 {
                     TRACE_T0();
-                    ok = mbar_wait(smem_u32(&bars.acc_empty[a]), apar, abort_flag, p.status, 4);
-                    TRACE_ADD(1);
+                    ok = mbar_wait(empty0 + 8 * s, par, abort_flag, p.status, 1);
+                    TRACE_ADD(0);
+                }
+                if (!ok) break;
+                const uint32_t full = full0 + 8 * s;
+                const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
+                if (p.shifted) {
+                    if (elect_one()) {
+                        mbar_expect_tx(full, (uint32_t)(p.a_rows * CH));
+                        tma_load_2d(st, &map_a, 0, row0, full);
+                    }
+                } else if (elect_one()) {
+                    mbar_expect_tx(full, (uint32_t)stage_bytes);
+                    for (int c = 0; c < G; ++c) {
+                        tma_load_2d(st + c * a_chunk_bytes, &map_a, p.col_off[j + c],
+                                    row0 + p.row_off[j + c], full);
+                        if (!RESIDENT_B)
+                            tma_load_2d(st + G * a_chunk_bytes + c * b_tile_bytes, &map_b, 0,
+                                        (j + c) * p.n_total + brow0, full);
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp <= kMmaWarps) {
+        // ------------------------------------------------------------- MMA issuers (warps 1..4)
+        const int mw = warp - 1;
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) |
+                               ((uint32_t)(p.n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+        // descriptor = constant upper word | (address >> 4) in the lower word
+        const uint64_t desc_hi =
+            (uint64_t)(((uint32_t)(8 * CH) >> 4) | (1u << 14) |
+                       ((CH == 128 ? 2u : (CH == 64 ? 4u : 6u)) << 29)) << 32;
+        const uint32_t desc_lo_flags = 1u << 16;
+        const int k_steps = CH / 32;
+        bool ok = true;
+        if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
+        for (int i = mw; i < my_tiles && ok && mw < n_mma; i += n_mma) {
+            const int a = i % n_acc;
+            const uint32_t apar = ((i / n_acc) & 1) ^ 1;
+            {
+                TRACE_T0();
+                ok = mbar_wait(acc_empty0 + 8 * a, apar, abort_flag, p.status, 4);
+                TRACE_ADD(1);
+            }
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
+            for (int gi = 0; gi < n_groups; ++gi) {
+                const int lslot = (i / n_mma) * n_groups + gi;
+                const int s = mw + n_mma * (lslot % ring);
+                const uint32_t par = (lslot / ring) & 1;
+                const int j = gi * G;
+                {
+                    TRACE_T0();
+                    ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8);
+                    TRACE_ADD(2);
                 }
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
-                uint32_t accumulate = 0;
-                for (int gi = 0, j = 0; gi < n_groups; ++gi) {
-                    {
-                        TRACE_T0();
-                        ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8);
-                        TRACE_ADD(2);
+                const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
+                if (elect_one()) {
+                    for (int c = 0; c < G; ++c) {
+                        const uint32_t a_addr = p.shifted ? st + p.row_off[j + c] * CH
+                                                          : st + c * a_chunk_bytes;
+                        const uint32_t a_lo = (a_addr >> 4) | desc_lo_flags;
+                        const uint32_t b_addr = RESIDENT_B ? resident_addr + (j + c) * b_tile_bytes
+                                                           : st + G * a_chunk_bytes + c * b_tile_bytes;
+                        const uint32_t b_lo = (b_addr >> 4) | desc_lo_flags;
+                        for (int k = 0; k < k_steps; ++k)
+                            mma_i8(d_tmem, desc_hi | (a_lo + 2 * k), desc_hi | (b_lo + 2 * k), idesc,
+                                   (uint32_t)(gi | c | k));
                     }
-                    if (!ok) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
-                    if (elect_one()) {
-                        for (int c = 0; c < G; ++c) {
-                            const uint32_t a_lo = ((st + c * a_chunk_bytes) >> 4) | desc_lo_flags;
-                            const uint32_t b_addr = RESIDENT_B
-                                                        ? resident_addr + (j + c) * b_tile_bytes
-                                                        : st + G * a_chunk_bytes + c * b_tile_bytes;
-                            const uint32_t b_lo = (b_addr >> 4) | desc_lo_flags;
-                            for (int k = 0; k < k_steps; ++k) {
-                                mma_i8(d_tmem, desc_hi | (a_lo + 2 * k), desc_hi | (b_lo + 2 * k),
-                                       idesc, accumulate | c | k);
-                            }
-                        }
-                        mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
-                    }
-                    __syncwarp();
-                    accumulate = 1;
-                    j += G;
-                    if (++s == n_stages) {
-                        s = 0;
-                        par ^= 1;
-                    }
+                    mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
                 }
-                if (ok && elect_one()) mma_commit(smem_u32(&bars.acc_full[a]));
                 __syncwarp();
-                if (++a == n_acc) {
-                    a = 0;
-                    apar ^= 1;
-                }
             }
+            if (ok && elect_one()) mma_commit(acc_full0 + 8 * a);
+            __syncwarp();
         }
     } else {
-        // ------------------------------------------------------------- epilogue (warps 2..17)
+        // ------------------------------------------------------------- epilogue (warps 5..20)
         const int q = warp & 3;         // this warp's quarter of tensor memory
-        const int wg = (warp - 2) >> 2;  // epilogue warpgroup
+        const int wg = (warp - 1 - kMmaWarps) >> 2;  // epilogue warpgroup
         const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
         const int c_begin = p.split_cols ? wg * c_span : 0;
         const int c_end = c_begin + c_span;
@@ -372,7 +379,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             {
                 TRACE_T0();
                 ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
-                if (threadIdx.x == 64) TRACE_ADD(3);
+                if (threadIdx.x == 32 * (1 + kMmaWarps)) TRACE_ADD(3);
             }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -440,8 +447,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 
 #ifdef ACCERL_TC_TRACE
-    if (lane == 0 && (warp == 0 || warp == 1 || warp == 2))
-        atomicAdd((unsigned long long *)(p.status + 16) + p.trace_slot * 8 + 4 + warp,
+    if (lane == 0 && (warp == 0 || warp == 1 || warp == 1 + kMmaWarps))
+        atomicAdd((unsigned long long *)(p.status + 16) + p.trace_slot * 8 + 4 + (warp > 1 ? 2 : warp),
                   (unsigned long long)(clock64() - trace_start));
 #endif
     // ---------------------------------------------------------------- teardown
@@ -512,19 +519,26 @@ size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
 {
     const int a_chunk = kTileM * p.chunk_bytes, b_tile = p.n_tile * p.chunk_bytes;
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
-    return 1024 + res + (size_t)p.n_stages * p.group * (a_chunk + (resident_b ? 0 : b_tile));
+    const size_t stage = p.shifted ? (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
+                                   : (size_t)p.group * (a_chunk + (resident_b ? 0 : b_tile));
+    return 1024 + res + (size_t)p.n_stages * stage;
 }
 
 // Choose ring sizes for a problem; returns false if even the smallest pipeline does not fit.
 bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
 {
     const size_t limit = 216 * 1024;  // leaves room for the static shared variables
-    // chunks per stage: the largest divisor of n_chunks that keeps a stage at or under 32 KB
+    // chunks per stage: the largest divisor of n_chunks that keeps a stage at or under 16 KB
     const int per_chunk = kTileM * p.chunk_bytes + (resident_b ? 0 : p.n_tile * p.chunk_bytes);
     p.group = 1;
     for (int g = 1; g <= p.n_chunks; ++g)
-        if (p.n_chunks % g == 0 && g * per_chunk <= 32 * 1024) p.group = g;
-    for (int s = kTcMaxStages; s >= 2; --s) {
+        if (p.n_chunks % g == 0 && g * per_chunk <= 16 * 1024) p.group = g;
+    {
+        const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
+        p.n_acc_stages = std::min(kTcMaxAccStages, 512 / acc_cols);
+        p.n_mma = std::min(kMmaWarps, p.n_acc_stages);
+    }
+    for (int s = kTcMaxStages / p.n_mma * p.n_mma; s >= p.n_mma && s >= 2; s -= p.n_mma) {
         p.n_stages = s;
         if (tc_smem_bytes(p, resident_b) <= limit) {
             const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;

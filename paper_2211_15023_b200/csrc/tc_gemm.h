@@ -8,8 +8,8 @@
 namespace accerl {
 
 constexpr int kTcMaxChunks = 64;
-constexpr int kTcMaxStages = 8;
-constexpr int kTcMaxAccStages = 4;
+constexpr int kTcMaxStages = 12;
+constexpr int kTcMaxAccStages = 8;
 constexpr int kTcMaxN = 512;
 
 struct TcGemmParams {
@@ -21,6 +21,10 @@ struct TcGemmParams {
     int m_tiles, n_tiles, n_tile, n_total;
     int n_stages, n_acc_stages, tmem_cols;
     int group;  // K chunks per shared-memory stage
+    int n_mma;  // MMA-issuing warps in use
+    // shifted = 1: every chunk reads the same columns at a different row offset, so one TMA box of
+    // a_rows = 128 + max(row_off) rows per tile serves all of them (needs resident weights)
+    int shifted, a_rows;
     // GEMM row -> output position: row = n * rows_per_image + Y * grid_w + X, kept when
     // Y < out_h and X < out_w; stored at row n * out_rows_per_image + (Y/s) * out_grid_w + X/s,
     // byte ((Y%s) * s + X%s) * n_total + channel, rows `out_pitch` bytes apart (s = out_s2d)

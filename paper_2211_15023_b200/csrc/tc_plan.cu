@@ -164,6 +164,8 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             row_bytes = CH;
             g.rows_per_image = Hs * Ws;
             g.grid_w = Ws;
+            g.shifted = 1;
+            g.a_rows = round_up(128 + (t - 1) * Ws + (t - 1), 8);
             packed.assign((size_t)g.n_chunks * n_total * CH, 0);
             for (int by = 0; by < t; ++by)
                 for (int bx = 0; bx < t; ++bx) {
@@ -222,8 +224,14 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         g.trace_slot = (int)p->tc_steps.size();
         // resident weights when the whole matrix fits beside a useful pipeline
         ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * g.chunk_bytes <= 96 * 1024;
+        if (g.shifted && (!ts.resident_b || g.a_rows > 256)) {
+            g.shifted = 0;  // fall back to one box per tap
+            g.a_rows = 128;
+        }
         if (!tc_choose_pipeline(g, ts.resident_b)) {
             ts.resident_b = false;
+            g.shifted = 0;
+            g.a_rows = 128;
             if (!tc_choose_pipeline(g, false)) {  // generic plan stays
                 p->tensor_s2d.assign(n_layers + 1, 1);
                 p->tc_steps.clear();
@@ -234,8 +242,8 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         accerl_status st = upload_bytes(p, packed.data(), packed.size(), &w_dev);
         if (st != ACCERL_OK) return st;
         const long long rows = (long long)p->max_batch * rows_in_per_image;
-        st = tc_make_map(ts.map_a, p->bufs[L.in_buf].ptr, rows, row_bytes, row_bytes, 128,
-                         g.chunk_bytes);
+        st = tc_make_map(ts.map_a, p->bufs[L.in_buf].ptr, rows, row_bytes, row_bytes,
+                         g.shifted ? g.a_rows : 128, g.chunk_bytes);
         if (st != ACCERL_OK) return st;
         st = tc_make_map(ts.map_b, w_dev, (long long)g.n_chunks * n_total, g.chunk_bytes,
                          g.chunk_bytes, g.n_tile, g.chunk_bytes);
