@@ -269,17 +269,28 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         __syncwarp();
         bool ok = true;
-        for (int i = 0; i < my_tiles && ok; ++i) {
-            const int t = blockIdx.x + i * gridDim.x;
-            const int mt = t / p.n_tiles, nt = t - mt * p.n_tiles;
+        // Ring position of the current tile inside its issuing warp's ring; all warps' rings
+        // advance in lockstep (n_groups slots per tile), so one running position serves.
+        int w = 0, base_slot = 0;
+        uint32_t base_phase = 0;
+        int t = blockIdx.x;
+        for (int i = 0; i < my_tiles && ok; ++i, t += gridDim.x) {
+            int mt = t, nt = 0;
+            if (p.n_tiles != 1) {
+                mt = t / p.n_tiles;
+                nt = t - mt * p.n_tiles;
+            }
             const int row0 = mt * kTileM, brow0 = nt * p.n_tile;
             for (int gi = 0; gi < n_groups; ++gi) {
                 const int j = gi * G;
-                // issuing warp i % n_mma owns every n_mma-th ring slot; within its slots this
-                // tile's group gi is local slot (i / n_mma) * n_groups + gi
-                const int lslot = (i / n_mma) * n_groups + gi;
-                const int s = (i % n_mma) + n_mma * (lslot % ring);
-                const uint32_t par = ((lslot / ring) & 1) ^ 1;
+                int sl = base_slot + gi;
+                uint32_t ph = base_phase;
+                while (sl >= ring) {
+                    sl -= ring;
+                    ph ^= 1;
+                }
+                const int s = w + n_mma * sl;
+                const uint32_t par = ph ^ 1;
                 {
                     TRACE_T0();
                     ok = mbar_wait(empty0 + 8 * s, par, abort_flag, p.status, 1);
@@ -305,6 +316,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 __syncwarp();
             }
+            if (++w == n_mma) {
+                w = 0;
+                base_slot += n_groups;
+                while (base_slot >= ring) {
+                    base_slot -= ring;
+                    base_phase ^= 1;
+                }
+            }
         }
     } else if (warp <= kMmaWarps) {
         // ------------------------------------------------------------- MMA issuers (warps 1..4)
@@ -319,9 +338,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int k_steps = CH / 32;
         bool ok = true;
         if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
+        int a = mw, base_slot = 0;
+        uint32_t aphase = 0, base_phase = 0;
         for (int i = mw; i < my_tiles && ok && mw < n_mma; i += n_mma) {
-            const int a = i % n_acc;
-            const uint32_t apar = ((i / n_acc) & 1) ^ 1;
+            const uint32_t apar = aphase ^ 1;
             {
                 TRACE_T0();
                 ok = mbar_wait(acc_empty0 + 8 * a, apar, abort_flag, p.status, 4);
@@ -331,9 +351,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
             for (int gi = 0; gi < n_groups; ++gi) {
-                const int lslot = (i / n_mma) * n_groups + gi;
-                const int s = mw + n_mma * (lslot % ring);
-                const uint32_t par = (lslot / ring) & 1;
+                int sl = base_slot + gi;
+                uint32_t par = base_phase;
+                while (sl >= ring) {
+                    sl -= ring;
+                    par ^= 1;
+                }
+                const int s = mw + n_mma * sl;
                 const int j = gi * G;
                 {
                     TRACE_T0();
@@ -361,6 +385,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             if (ok && elect_one()) mma_commit(acc_full0 + 8 * a);
             __syncwarp();
+            a += n_mma;
+            if (a >= n_acc) {
+                a -= n_acc;
+                aphase ^= 1;
+            }
+            base_slot += n_groups;
+            while (base_slot >= ring) {
+                base_slot -= ring;
+                base_phase ^= 1;
+            }
         }
     } else {
         // ------------------------------------------------------------- epilogue (warps 5..20)
@@ -373,9 +407,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
             if (!p.split_cols && (tile_i % kEpiGroups) != wg) continue;
-            const int mt = t / p.n_tiles, nt = t % p.n_tiles;
-            const int a = tile_i % n_acc;
-            const uint32_t apar = (tile_i / n_acc) & 1;
+            int mt = t, nt = 0;
+            if (p.n_tiles != 1) {
+                mt = t / p.n_tiles;
+                nt = t - mt * p.n_tiles;
+            }
+            const int a = tile_i & (n_acc - 1);  // n_acc is a power of two
+            const uint32_t apar = (tile_i >> p.n_acc_log2) & 1;
             {
                 TRACE_T0();
                 ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
@@ -385,62 +423,57 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int m = mt * kTileM + q * 32 + lane;
-            // which output position is this GEMM row?
-            const int n = m / p.rows_per_image;
-            const int r = m - n * p.rows_per_image;
-            const int Y = r / p.grid_w, X = r - Y * p.grid_w;
+            // which output position is this GEMM row?  Division-free: a float estimate of
+            // m / rows_per_image corrected by stepping, a 16.16 reciprocal for the row inside the image
+            // (exact for r < 65536), shifts for the power-of-two space-to-depth factor.
+            int n = __float2int_rz(__int2float_rn(m) * p.inv_rows_per_image);
+            int r = m - n * p.rows_per_image;
+            while (r < 0) {
+                --n;
+                r += p.rows_per_image;
+            }
+            while (r >= p.rows_per_image) {
+                ++n;
+                r -= p.rows_per_image;
+            }
+            const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
             const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
-            const int s2 = p.out_s2d;
+            const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
             const long long out_row =
-                (long long)n * p.out_rows_per_image + (Y / s2) * p.out_grid_w + X / s2;
+                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh);
             const int col0 = nt * p.n_tile;
-            int8_t *dst = p.out + out_row * p.out_pitch + ((Y % s2) * s2 + X % s2) * p.n_total + col0;
+            int8_t *dst = p.out + out_row * p.out_pitch +
+                          ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
             float *ldst = p.logits_mode ? p.logits + (long long)m * p.n_actions : nullptr;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_cols);
-            for (int c0 = c_begin; c0 < c_end; c0 += 32) {
-                const bool two = c0 + 32 <= c_end;  // 32 columns per round, 16 for a narrow tail
-                int acc[32];
-                if (two) {
-                    tmem_ld32(taddr + c0, acc);
-                } else {
-                    int lo[16];
-                    tmem_ld16(taddr + c0, lo);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) acc[i] = lo[i];
-                }
+            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+                int acc[16];
+                tmem_ld16(taddr + c0, acc);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c0 + 32 >= c_end) {
+                if (c0 + 16 >= c_end) {
                     // all of this warp's reads of the stage are done: hand it back to the MMA warp
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars.acc_empty[a]));
+                    if (lane == 0) mbar_arrive(acc_empty0 + 8 * a);
                 }
                 if (!valid) continue;
+                float ks[16], bs[16];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (h == 1 && !two) break;
-                    const int cc = c0 + 16 * h;
-                    int part[16];
-                    float ks[16], bs[16];
+                for (int g = 0; g < 4; ++g) {
+                    const float4 kv = *reinterpret_cast<const float4 *>(&s_ks[col0 + c0 + 4 * g]);
+                    const float4 bv = *reinterpret_cast<const float4 *>(&s_bs[col0 + c0 + 4 * g]);
+                    ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                    bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+                }
+                if (ldst) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) part[i] = acc[16 * h + i];
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const float4 kv = *reinterpret_cast<const float4 *>(&s_ks[col0 + cc + 4 * g]);
-                        const float4 bv = *reinterpret_cast<const float4 *>(&s_bs[col0 + cc + 4 * g]);
-                        ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
-                        bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
-                    }
-                    if (ldst) {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            if (col0 + cc + i < p.n_actions)
-                                ldst[col0 + cc + i] = epilogue_float(part[i], ks[i], bs[i], false);
-                    } else {
-                        uint32_t w[4];
-                        requant16(part, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
-                        *reinterpret_cast<uint4 *>(dst + cc) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
+                    for (int i = 0; i < 16; ++i)
+                        if (col0 + c0 + i < p.n_actions)
+                            ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
+                } else {
+                    uint32_t w[4];
+                    requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
+                    *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         }
@@ -524,6 +557,13 @@ size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
     return 1024 + res + (size_t)p.n_stages * stage;
 }
 
+static int pow2_floor(int v)
+{
+    int r = 1;
+    while (2 * r <= v) r *= 2;
+    return r;
+}
+
 // Choose ring sizes for a problem; returns false if even the smallest pipeline does not fit.
 bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
 {
@@ -535,17 +575,18 @@ bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
         if (p.n_chunks % g == 0 && g * per_chunk <= 16 * 1024) p.group = g;
     {
         const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
-        p.n_acc_stages = std::min(kTcMaxAccStages, 512 / acc_cols);
+        p.n_acc_stages = pow2_floor(std::min(kTcMaxAccStages, 512 / acc_cols));
         p.n_mma = std::min(kMmaWarps, p.n_acc_stages);
     }
     for (int s = kTcMaxStages / p.n_mma * p.n_mma; s >= p.n_mma && s >= 2; s -= p.n_mma) {
         p.n_stages = s;
         if (tc_smem_bytes(p, resident_b) <= limit) {
             const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
-            p.n_acc_stages = std::min(kTcMaxAccStages, 512 / acc_cols);
+            p.n_acc_stages = pow2_floor(std::min(kTcMaxAccStages, 512 / acc_cols));
             int cols = 32;
             while (cols < p.n_acc_stages * acc_cols) cols *= 2;
             p.tmem_cols = cols;
+            p.n_acc_log2 = p.n_acc_stages == 8 ? 3 : (p.n_acc_stages == 4 ? 2 : (p.n_acc_stages == 2 ? 1 : 0));
             return true;
         }
     }

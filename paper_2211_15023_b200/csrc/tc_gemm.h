@@ -19,7 +19,7 @@ struct TcGemmParams {
     int row_off[kTcMaxChunks], col_off[kTcMaxChunks];
     // tiling
     int m_tiles, n_tiles, n_tile, n_total;
-    int n_stages, n_acc_stages, tmem_cols;
+    int n_stages, n_acc_stages, n_acc_log2, tmem_cols;
     int group;  // K chunks per shared-memory stage
     int n_mma;  // MMA-issuing warps in use
     // shifted = 1: every chunk reads the same columns at a different row offset, so one TMA box of
@@ -30,6 +30,9 @@ struct TcGemmParams {
     // byte ((Y%s) * s + X%s) * n_total + channel, rows `out_pitch` bytes apart (s = out_s2d)
     int batch, rows_per_image, grid_w, out_h, out_w;
     int out_s2d, out_rows_per_image, out_grid_w, out_pitch;
+    int out_s2d_log2;
+    float inv_rows_per_image;  // 1 / rows_per_image, for the division-free row decode
+    unsigned grid_w_magic;     // ceil(2^32 / grid_w)
     // epilogue
     const float *kscale, *bias;
     float s_out, inv_s_out;

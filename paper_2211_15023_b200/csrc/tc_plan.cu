@@ -94,6 +94,7 @@ bool conv_fits(const accerl_layer_desc &d)
     const int t = d.kh / d.stride;
     if (t * t > kTcMaxChunks) return false;
     if (d.out_c % 16 || d.out_c > 256) return false;
+    if (d.stride != 1 && d.stride != 2 && d.stride != 4) return false;
     if (d.skip_from >= 0) return false;
     return true;
 }
@@ -205,6 +206,9 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         g.out_w = L.out_w;
         const int so = p->tensor_s2d[i + 1];
         g.out_s2d = so;
+        g.out_s2d_log2 = so == 4 ? 2 : (so == 2 ? 1 : 0);
+        g.inv_rows_per_image = 1.0f / (float)g.rows_per_image;
+        g.grid_w_magic = g.grid_w == 1 ? 0xffffffffu : (unsigned)(((1ULL << 32) + g.grid_w - 1) / g.grid_w);
         g.out_rows_per_image = (L.out_h / so) * (L.out_w / so);
         g.out_grid_w = L.out_w / so;
         g.out_pitch = so * so * n_total;
