@@ -281,7 +281,8 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
         case Step::INGEST_S2D:
             ACCERL_CUDA_TRY(launch_ingest_u8_s2d((const uint8_t *)obs_dev, p->lut,
                                                  p->bufs[p->layers[0].in_buf].ptr, B, p->in_c,
-                                                 p->in_h, p->in_w, p->tensor_s2d[0], st));
+                                                 p->in_h, p->in_w, p->tensor_s2d[0], p->ingest_arith,
+                                                 p->ingest_mul, p->ingest_add, st));
             break;
         case Step::TC_GEMM: {
             TcStep &t = p->tc_steps[s.tc];
@@ -502,6 +503,7 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
             lut[u] = (int8_t)r;
         }
         if ((st = upload(p, lut, &p->lut)) != ACCERL_OK) return fail(st);
+        p->ingest_arith = fit_ingest_line(lut.data(), &p->ingest_mul, &p->ingest_add) ? 1 : 0;
     }
     {
         std::vector<int> zero(256, 0);  // word 0 is the status; the rest is trace space

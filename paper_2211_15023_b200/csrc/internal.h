@@ -86,6 +86,8 @@ struct accerl_policy {
     int sm_count = 0;
     std::vector<accerl::DeviceBuf> bufs;  // bufs[0] holds the quantised input
     int8_t *lut = nullptr;                // device, 256-entry uint8 -> int8 input table
+    int ingest_arith = 0;                 // the table is the line min((u * mul + add) >> 24, 127)
+    uint32_t ingest_mul = 0, ingest_add = 0;
     int *status_word = nullptr;           // device, set by kernels whose bounded waits give up
     size_t workspace_bytes = 0;
     std::vector<void *> owned;            // every device allocation, for destroy

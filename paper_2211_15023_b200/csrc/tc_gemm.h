@@ -55,6 +55,8 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
 
 // uint8 NCHW frames -> int8 space-to-depth(s) rows [B * (H/s) * (W/s)][s*s*C]
 cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
-                                 int H, int W, int s, cudaStream_t st);
+                                 int H, int W, int s, int arith, uint32_t mul, uint32_t add,
+                                 cudaStream_t st);
+bool fit_ingest_line(const int8_t *lut, uint32_t *mul, uint32_t *add);
 
 }  // namespace accerl

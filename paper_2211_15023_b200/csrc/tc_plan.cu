@@ -3,48 +3,69 @@
 // parameters.  Also holds the input kernel that writes frames in space-to-depth form.
 #include <string.h>
 
+#include <algorithm>
+
 #include "epilogue.cuh"
 #include "internal.h"
 
 namespace accerl {
 
 // ---------------------------------------------------------------------------------------
-// uint8 NCHW frames -> int8 space-to-depth(s) rows, C = 4, s = 4: each thread turns one
-// 4-pixel run of all four channel planes into 16 output bytes ((dx, c) order).
+// uint8 NCHW frames -> int8 space-to-depth(s) rows, C = 4, s = 4: each thread turns one 4 x 4
+// pixel block of all four channel planes into one 64-byte output row ((dy, dx, c) order).
+// With ARITH the table lookup is replaced by q = min((u * mul + add) >> 24, 127), a fixed-point
+// line that the host has checked against all 256 table entries; the product fits 32 bits, so the
+// code is simply the top byte of the multiply-add.
 // ---------------------------------------------------------------------------------------
+template <bool ARITH>
 __global__ void ingest_u8_s2d44_kernel(const uint8_t *__restrict__ obs,
                                        const int8_t *__restrict__ lut, uint4 *__restrict__ out,
-                                       long long total, int H, int W)
+                                       long long total, int H, int W, uint32_t mul, uint32_t add)
 {
     __shared__ int8_t s_lut[256];
-    for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = lut[i];
-    __syncthreads();
+    if (!ARITH) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = lut[i];
+        __syncthreads();
+    }
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
     const int Ws = W / 4, Hs = H / 4;
-    // idx = ((n * Hs + Y) * 4 + dy) * Ws + X
+    // one thread = one output row (n, Y, X): sixteen independent 4-byte loads (4 image rows of 4
+    // channel planes) are in flight before the first is used, then 64 contiguous bytes are stored
     int X = (int)(idx % Ws);
     long long t = idx / Ws;
-    int dy = (int)(t % 4);
-    t /= 4;
     int Y = (int)(t % Hs);
     long long n = t / Hs;
-    uint32_t plane[4];
+    uint32_t plane[4][4];  // [dy][c]
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
-        plane[c] = *reinterpret_cast<const uint32_t *>(
-            obs + ((n * 4 + c) * H + 4 * Y + dy) * W + 4 * X);
-    uint32_t w[4];
-#pragma unroll
-    for (int dx = 0; dx < 4; ++dx) {
-        uint32_t word = 0;
+    for (int dy = 0; dy < 4; ++dy)
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            word |= (uint32_t)(uint8_t)s_lut[(plane[c] >> (8 * dx)) & 0xff] << (8 * c);
-        w[dx] = word;
+            plane[dy][c] = __ldg(reinterpret_cast<const uint32_t *>(
+                obs + ((n * 4 + c) * H + 4 * Y + dy) * W + 4 * X));
+#pragma unroll
+    for (int dy = 0; dy < 4; ++dy) {
+        uint32_t w[4];
+#pragma unroll
+        for (int dx = 0; dx < 4; ++dx) {
+            if (ARITH) {
+                uint32_t pr[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) pr[c] = ((plane[dy][c] >> (8 * dx)) & 0xff) * mul + add;
+                // top bytes of the four products, channel 0 in the low byte
+                const uint32_t lo = __byte_perm(pr[0], pr[1], 0x0073);
+                const uint32_t hi = __byte_perm(pr[2], pr[3], 0x0073);
+                w[dx] = __vminu4(__byte_perm(lo, hi, 0x5410), 0x7f7f7f7fu);
+            } else {
+                uint32_t word = 0;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    word |= (uint32_t)(uint8_t)s_lut[(plane[dy][c] >> (8 * dx)) & 0xff] << (8 * c);
+                w[dx] = word;
+            }
+        }
+        out[idx * 4 + dy] = make_uint4(w[0], w[1], w[2], w[3]);
     }
-    // row (n, Y, X) of 64 bytes, this thread's 16 bytes start at dy * 16
-    out[((n * Hs + Y) * Ws + X) * 4 + dy] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // any C, s: one thread per output byte
@@ -65,13 +86,60 @@ __global__ void ingest_u8_s2d_any_kernel(const uint8_t *__restrict__ obs,
     out[idx] = lut[obs[((n * C + c) * H + s * Y + dy) * W + s * X + dx]];
 }
 
+// Fit q(u) = min((u * mul + add) >> 24, 127) to a 256-entry input table; false if no line fits.
+bool fit_ingest_line(const int8_t *lut, uint32_t *mul, uint32_t *add)
+{
+    int last = 255;  // entries from the first 127 on may be clamped
+    for (int u = 0; u < 256; ++u) {
+        if (lut[u] < 0) return false;
+        if (lut[u] == 127) {
+            last = u;
+            break;
+        }
+    }
+    if (last < 2) return false;
+    const long long one = 1LL << 24;
+    const double slope = (double)lut[last] / last;
+    const long long a0 = (long long)(slope * one);
+    for (long long a = a0 - 4096; a <= a0 + 4096; ++a) {
+        if (a <= 0) continue;
+        long long lo = 0, hi = one * 256;  // add in [lo, hi)
+        for (int u = 0; u < 256 && lo < hi; ++u) {
+            const long long q = lut[u];
+            lo = std::max(lo, q * one - u * a);
+            if (u < last) hi = std::min(hi, (q + 1) * one - u * a);
+        }
+        hi = std::min(hi, (1LL << 32) - 255 * a);  // the multiply-add must not wrap
+        if (lo < hi) {
+            const long long b = lo + (hi - lo) / 2;
+            bool ok = true;
+            for (int u = 0; u < 256 && ok; ++u) {
+                const unsigned long long v = (unsigned long long)u * a + b;
+                ok = v < (1ULL << 32) && std::min<long long>((long long)(v >> 24), 127) == lut[u];
+            }
+            if (ok) {
+                *mul = (uint32_t)a;
+                *add = (uint32_t)b;
+                return true;
+            }
+        }
+    }
+    return false;
+}
+
 cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
-                                 int H, int W, int s, cudaStream_t st)
+                                 int H, int W, int s, int arith, uint32_t mul, uint32_t add,
+                                 cudaStream_t st)
 {
     if (C == 4 && s == 4 && W % 4 == 0) {
-        long long total = (long long)B * H * (W / 4);
-        ingest_u8_s2d44_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(
-            obs, lut, (uint4 *)out, total, H, W);
+        long long total = (long long)B * (H / 4) * (W / 4);
+        const unsigned blocks = (unsigned)((total + 255) / 256);
+        if (arith)
+            ingest_u8_s2d44_kernel<true><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, H, W,
+                                                                mul, add);
+        else
+            ingest_u8_s2d44_kernel<false><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, H, W,
+                                                                 mul, add);
     } else {
         long long total = (long long)B * C * H * W;
         ingest_u8_s2d_any_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(obs, lut, out, total,
