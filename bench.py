@@ -236,7 +236,10 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(W.CONFIGS))
     ap.add_argument("--ref-sample", type=int, default=256)
-    ap.add_argument("--cpu-sample", type=int, default=512)
+    ap.add_argument("--cpu-sample", type=int, default=2048)
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the workload's batch (profiling captures on a small case only)")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-others", action="store_true", help="skip the brief runs of other workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -258,7 +261,7 @@ def main() -> None:
     torch.cuda.set_device(local)
 
     name = args.workload
-    batch = W.config(name)["batch"]
+    batch = args.batch or W.config(name)["batch"]
     in_bytes = W.input_bytes_per_state(name) * batch
     n_buffers = 3 if in_bytes * 3 < (8 << 30) else 2
     r = time_workload(P, torch, name, batch, args.steps, args.warmup, n_buffers, local, dist,
@@ -342,16 +345,18 @@ def main() -> None:
             o["policy"].close()
 
     # ---- CPU oracle on a bounded sample of the same workload (reported baseline)
-    import oracle
-    sample = min(batch, args.cpu_sample)
-    pol = W.drawn_int8_policy(name)
-    so, su = W.observations(name, sample), W.uniforms(name, sample)
-    oracle.forward(pol, so[:8], su[:8], keep=False)
-    t0 = time.perf_counter()
-    oracle.forward(pol, so, su, keep=False)
-    cpu_dt = time.perf_counter() - t0
-    cpu = dict(value=sample / cpu_dt, unit=UNIT, cores=os.cpu_count(), kind="oracle",
-               sample="first %d states of the %d-state batch, one pass" % (sample, batch))
+    cpu = None
+    if not args.no_cpu:
+        import oracle
+        sample = min(batch, args.cpu_sample)
+        pol = W.drawn_int8_policy(name)
+        so, su = W.observations(name, sample), W.uniforms(name, sample)
+        oracle.forward(pol, so[:8], su[:8], keep=False)
+        t0 = time.perf_counter()
+        oracle.forward(pol, so, su, keep=False)
+        cpu_dt = time.perf_counter() - t0
+        cpu = dict(value=sample / cpu_dt, unit=UNIT, cores=os.cpu_count(), kind="oracle",
+                   sample="first %d states of the %d-state batch, one pass" % (sample, batch))
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
