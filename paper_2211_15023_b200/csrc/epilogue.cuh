@@ -78,4 +78,45 @@ __device__ __forceinline__ void requant16(const int (&acc)[16], const float (&ks
     for (int g = 0; g < 4; ++g) w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
 }
 
+// One requantised code by the three-step division: t = y * r, e = y - s * t (exact in one fma),
+// d = t + e * r.  With r = fl(1 / s) this is the classical correctly rounded quotient except for
+// rare operand patterns, so it is only used for scales for which fastdiv_code() has been compared
+// with exact_code() over every fp32 value y can take (see verify_fastdiv in tc_plan.cu).  ReLU
+// is applied to the quotient, which has the sign of y; the saturating pack does the clamp.
+template <bool RELU>
+__device__ __forceinline__ int fastdiv_rint(float y, float s, float r)
+{
+    const float t = __fmul_rn(y, r);
+    const float e = __fmaf_rn(-s, t, y);
+    float d = __fmaf_rn(e, r, t);
+    if (RELU) d = fmaxf(d, 0.f);  // the quotient has the sign of y
+    return __float2int_rn(d);
+}
+
+// the defining expression, for one element: clamp(rintf(max?(y) / s), -128, 127)
+__device__ __forceinline__ int exact_code(float y, float s, bool relu)
+{
+    if (relu) y = fmaxf(y, 0.f);
+    return (int)requant(y, s);
+}
+
+template <bool RELU>
+__device__ __forceinline__ int fastdiv_code(float y, float s, float r)
+{
+    return min(max(fastdiv_rint<RELU>(y, s, r), -128), 127);  // what the saturating pack does
+}
+
+template <bool RELU>
+__device__ __forceinline__ void requant16_fastdiv(const int (&acc)[16], const float (&ks)[16],
+                                                  const float (&bs)[16], float s_out,
+                                                  float inv_s_out, uint32_t (&w)[4])
+{
+    int q[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+        q[i] = fastdiv_rint<RELU>(__fmaf_rn(__int2float_rn(acc[i]), ks[i], bs[i]), s_out, inv_s_out);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
+}
+
 }  // namespace accerl

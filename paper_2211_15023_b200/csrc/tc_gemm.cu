@@ -88,6 +88,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(32);  // polling warps must not take issue slots from the working ones
         if (*abort_flag) return false;
         if (clock64() - t0 > kWaitLimitCycles) {
             *abort_flag = 1;
@@ -472,7 +473,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
                 } else {
                     uint32_t w[4];
-                    requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
+                    if (p.fast_div) {
+                        if (p.relu_out) requant16_fastdiv<true>(acc, ks, bs, p.s_out, p.inv_s_out, w);
+                        else requant16_fastdiv<false>(acc, ks, bs, p.s_out, p.inv_s_out, w);
+                    } else {
+                        requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
+                    }
                     *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }

@@ -36,6 +36,7 @@ struct TcGemmParams {
     // epilogue
     const float *kscale, *bias;
     float s_out, inv_s_out;
+    int fast_div;  // 1: the three-step division has been verified for this s_out (epilogue.cuh)
     int relu_out;
     int split_cols;  // 1: both epilogue warpgroups share a tile (half the columns each)
     int8_t *out;
@@ -57,6 +58,8 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
 cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
                                  int H, int W, int s, int arith, uint32_t mul, uint32_t add,
                                  cudaStream_t st);
+// exhaustive check of the three-step division against the IEEE divide for one output scale
+accerl_status verify_fastdiv(float s_out, float inv_s_out, bool relu, float y_max, bool *ok);
 bool fit_ingest_line(const int8_t *lut, uint32_t *mul, uint32_t *add);
 
 }  // namespace accerl

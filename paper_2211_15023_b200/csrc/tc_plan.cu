@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 
 #include "epilogue.cuh"
 #include "internal.h"
@@ -149,6 +150,59 @@ cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *
 }
 
 // ---------------------------------------------------------------------------------------
+// exhaustive verification of the fast division for one output scale
+// ---------------------------------------------------------------------------------------
+template <bool RELU>
+__global__ void verify_fastdiv_kernel(float s, float r, float y_max, unsigned long long *bad)
+{
+    const unsigned long long total = 1ULL << 32;
+    unsigned long long mine = 0;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (unsigned long long)gridDim.x * blockDim.x) {
+        const float y = __uint_as_float((unsigned)i);
+        if (!(fabsf(y) <= y_max)) continue;  // also skips NaN
+        if (fastdiv_code<RELU>(y, s, r) != exact_code(y, s, RELU)) ++mine;
+    }
+    if (mine) atomicAdd(bad, mine);
+}
+
+// Compares fastdiv_code with the defining expression for every float |y| <= y_max.  Results are
+// remembered per (scale, relu, range) so that a scale is checked once per process.
+accerl_status verify_fastdiv(float s_out, float inv_s_out, bool relu, float y_max, bool *ok)
+{
+    struct Key {
+        float s, ymax;
+        bool relu, ok;
+    };
+    static std::vector<Key> cache;
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lock(mu);
+    for (const Key &k : cache)
+        if (k.s == s_out && k.relu == relu && k.ymax >= y_max) {
+            *ok = k.ok;
+            return ACCERL_OK;
+        }
+    *ok = false;
+    unsigned long long *bad = nullptr, host = 1;
+    ACCERL_CUDA_TRY(cudaMalloc(&bad, sizeof(*bad)));
+    cudaError_t e = cudaMemset(bad, 0, sizeof(*bad));
+    if (e == cudaSuccess) {
+        if (relu) verify_fastdiv_kernel<true><<<148 * 8, 256>>>(s_out, inv_s_out, y_max, bad);
+        else verify_fastdiv_kernel<false><<<148 * 8, 256>>>(s_out, inv_s_out, y_max, bad);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(&host, bad, sizeof(host), cudaMemcpyDeviceToHost);
+    cudaFree(bad);
+    if (e != cudaSuccess) {
+        set_error("verify_fastdiv: %s", cudaGetErrorString(e));
+        return ACCERL_ERR_CUDA;
+    }
+    *ok = host == 0;
+    cache.push_back(Key{s_out, y_max, relu, *ok});
+    return ACCERL_OK;
+}
+
+// ---------------------------------------------------------------------------------------
 // plan
 // ---------------------------------------------------------------------------------------
 
@@ -283,12 +337,25 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         g.kscale = L.kscale;
         g.bias = L.bias;
         g.s_out = L.s_out;
+        g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
         {
             volatile float inv = 1.0f / L.s_out;  // IEEE reciprocal, rounded once
             g.inv_s_out = inv;
         }
+        if (!logits) {
+            // largest |y| = |fma(acc, k, b)| the layer can produce: |acc| < 2^31
+            float kmax = 0.f, bmax = 0.f;
+            for (int c = 0; c < d.out_c; ++c) {
+                kmax = std::max(kmax, d.s_in * d.s_w[c]);
+                bmax = std::max(bmax, fabsf(d.bias[c]));
+            }
+            bool ok = false;
+            accerl_status vs = verify_fastdiv(g.s_out, g.inv_s_out, g.relu_out != 0,
+                                              2147483648.0f * kmax + bmax, &ok);
+            if (vs != ACCERL_OK) return vs;
+            g.fast_div = ok ? 1 : 0;
+        }
         g.split_cols = g.n_tile >= 128 ? 1 : 0;  // 128 / 256 columns: 32 / 64 per warpgroup
-        g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
         g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
         g.logits_mode = logits ? 1 : 0;
         g.n_actions = p->n_actions;
@@ -326,6 +393,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         s.layer = i;
         s.tc = (int)p->tc_steps.size() - 1;
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
+        if (g.fast_div) s.kernel += "[3-step divide verified]";
         s.covers = "layer " + std::to_string(i);
         steps.push_back(s);
     }

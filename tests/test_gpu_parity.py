@@ -178,6 +178,8 @@ def test_exact_ties_on_the_tensor_core_path():
     ref = oracle.forward(pol, obs, u)
     g = P.Policy(pol, b, flags=1)
     assert "tc_gemm" in g.info()["plan"]
+    # power-of-two scales are the easy case of the three-step division: it must have been verified
+    assert "3-step divide verified" in g.info()["plan"]
     out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
     compare(ref, *out, taps=g.read_activation)
     g.close()
