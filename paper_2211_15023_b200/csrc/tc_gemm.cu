@@ -196,6 +196,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ Barriers bars;
     __shared__ __align__(16) float s_ks[kTcMaxN], s_bs[kTcMaxN];
+    // per (chunk, k step): low descriptor words of the A and B operands, relative to the stage
+    // (B absolute when the weights are resident), so that the issue loop is a load and an add
+    __shared__ uint2 s_desc[kTcMaxChunks * 4];
     for (int i = threadIdx.x; i < p.n_total; i += blockDim.x) {
         s_ks[i] = p.kscale[i];
         s_bs[i] = p.bias[i];
@@ -214,6 +217,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;  // column stride of an accumulator stage
     volatile int *abort_flag = &bars.abort_flag;
 
+    {
+        const int ks_per_chunk = CH / 32;
+        const int Gt = p.shifted ? p.n_chunks : p.group;
+        for (int t = threadIdx.x; t < p.n_chunks * ks_per_chunk; t += blockDim.x) {
+            const int j = t / ks_per_chunk, k = t - j * ks_per_chunk, cl = j % Gt;
+            const uint32_t a_rel = (uint32_t)(p.shifted ? p.row_off[j] * CH : cl * a_chunk_bytes);
+            const uint32_t b_rel =
+                RESIDENT_B ? smem_u32(resident_b) + (uint32_t)(j * b_tile_bytes)
+                           : (uint32_t)(Gt * a_chunk_bytes + cl * b_tile_bytes);
+            s_desc[t] = make_uint2((a_rel >> 4) + 2 * k,
+                                   ((b_rel >> 4) + 2 * k) | (RESIDENT_B ? (1u << 16) : 0u));
+        }
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(smem_u32(&bars.full[s]), 1);
@@ -367,18 +383,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
+                const uint32_t st_lo = ((stages_addr + (uint32_t)s * stage_bytes) >> 4) | desc_lo_flags;
                 if (elect_one()) {
-                    for (int c = 0; c < G; ++c) {
-                        const uint32_t a_addr = p.shifted ? st + p.row_off[j + c] * CH
-                                                          : st + c * a_chunk_bytes;
-                        const uint32_t a_lo = (a_addr >> 4) | desc_lo_flags;
-                        const uint32_t b_addr = RESIDENT_B ? resident_addr + (j + c) * b_tile_bytes
-                                                           : st + G * a_chunk_bytes + c * b_tile_bytes;
-                        const uint32_t b_lo = (b_addr >> 4) | desc_lo_flags;
-                        for (int k = 0; k < k_steps; ++k)
-                            mma_i8(d_tmem, desc_hi | (a_lo + 2 * k), desc_hi | (b_lo + 2 * k), idesc,
-                                   (uint32_t)(gi | c | k));
+                    const int t0 = j * k_steps, t1 = t0 + G * k_steps;
+                    for (int t = t0; t < t1; ++t) {
+                        const uint2 rel = s_desc[t];
+                        const uint32_t b_lo = RESIDENT_B ? rel.y : st_lo + rel.y;
+                        mma_i8(d_tmem, desc_hi | (st_lo + rel.x), desc_hi | b_lo, idesc, (uint32_t)t);
                     }
                     mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
                 }
@@ -449,8 +460,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_cols);
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 int acc[16];
-                tmem_ld16(taddr + c0, acc);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                {
+                    TRACE_T0();
+                    tmem_ld16(taddr + c0, acc);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (threadIdx.x == 32 * (1 + kMmaWarps)) TRACE_ADD(7);
+                }
                 if (c0 + 16 >= c_end) {
                     // all of this warp's reads of the stage are done: hand it back to the MMA warp
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
