@@ -9,8 +9,8 @@
 // TMA box [128 rows][chunk bytes] fetched at (row0 + row_off[j], col_off[j]); rows whose window
 // would leave the image are computed and thrown away by the epilogue.
 //
-// Roles inside a CTA (672 threads): warp 0 issues TMA loads, warps 1..4 issue the MMAs (warp 1
-// owns the tensor-memory allocation), warps 5..20 are four epilogue warpgroups that drain accumulators (each warp its own
+// Roles inside a CTA (768 threads): warps 0..3 issue TMA loads, warps 4..7 issue the MMAs (warp 4
+// owns the tensor-memory allocation), warps 8..23 are four epilogue warpgroups that drain accumulators (each warp its own
 // 32-lane quarter of tensor memory), requantise and store; the warpgroups take tiles in turn,
 // or for wide tiles a quarter of the columns each.  The epilogue is latency bound per warp, so
 // four warps per scheduler are what keeps the issue slots busy.  The kernel is persistent: CTAs stride over the tile list, smem stages
@@ -31,7 +31,8 @@ namespace {
 constexpr int kTileM = 128;
 constexpr int kEpiGroups = 4;                       // epilogue warpgroups
 constexpr int kMmaWarps = 4;                        // MMA-issuing warps
-constexpr int kThreads = 32 * (1 + kMmaWarps) + 128 * kEpiGroups;
+constexpr int kProdWarps = kMmaWarps;                // TMA-issuing warps, one per MMA warp's ring
+constexpr int kThreads = 32 * (kProdWarps + kMmaWarps) + 128 * kEpiGroups;
 constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -244,7 +245,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == kProdWarps) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&bars.tmem_base)), "r"((uint32_t)p.tmem_cols)
                      : "memory");
@@ -276,22 +277,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int my_tiles = blockIdx.x < total_tiles
                              ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------- TMA producer
-        if (RESIDENT_B && elect_one()) {
-            mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
-            for (int j = 0; j < p.n_chunks; ++j)
-                tma_load_2d(resident_addr + j * b_tile_bytes, &map_b, 0, j * p.n_total,
-                            smem_u32(&bars.b_ready));
+    if (warp < kProdWarps) {
+        // ------------------------------------------------------------- TMA producers (warps 0..3)
+        // One wait -> arm -> load round trip takes several hundred cycles and cannot overlap
+        // with the next inside one warp, so every issuing warp's ring has a producer of its own.
+        const int pw = warp;
+        if (pw == 0) {
+            if (RESIDENT_B && elect_one()) {
+                mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)(p.n_chunks * b_tile_bytes));
+                for (int j = 0; j < p.n_chunks; ++j)
+                    tma_load_2d(resident_addr + j * b_tile_bytes, &map_b, 0, j * p.n_total,
+                                smem_u32(&bars.b_ready));
+            }
+            __syncwarp();
         }
-        __syncwarp();
         bool ok = true;
-        // Ring position of the current tile inside its issuing warp's ring; all warps' rings
-        // advance in lockstep (n_groups slots per tile), so one running position serves.
-        int w = 0, base_slot = 0;
+        int base_slot = 0;  // ring position of the current tile inside this warp's ring
         uint32_t base_phase = 0;
-        int t = blockIdx.x;
-        for (int i = 0; i < my_tiles && ok; ++i, t += gridDim.x) {
+        int t = blockIdx.x + pw * gridDim.x;
+        for (int i = pw; i < my_tiles && ok && pw < n_mma; i += n_mma, t += n_mma * gridDim.x) {
             int mt = t, nt = 0;
             if (p.n_tiles != 1) {
                 mt = t / p.n_tiles;
@@ -306,7 +310,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     sl -= ring;
                     ph ^= 1;
                 }
-                const int s = w + n_mma * sl;
+                const int s = pw + n_mma * sl;
                 const uint32_t par = ph ^ 1;
                 {
                     TRACE_T0();
@@ -333,18 +337,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 __syncwarp();
             }
-            if (++w == n_mma) {
-                w = 0;
-                base_slot += n_groups;
-                while (base_slot >= ring) {
-                    base_slot -= ring;
-                    base_phase ^= 1;
-                }
+            base_slot += n_groups;
+            while (base_slot >= ring) {
+                base_slot -= ring;
+                base_phase ^= 1;
             }
         }
-    } else if (warp <= kMmaWarps) {
-        // ------------------------------------------------------------- MMA issuers (warps 1..4)
-        const int mw = warp - 1;
+    } else if (warp < kProdWarps + kMmaWarps) {
+        // ------------------------------------------------------------- MMA issuers (warps 4..7)
+        const int mw = warp - kProdWarps;
         const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) |
                                ((uint32_t)(p.n_tile >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
         // descriptor = constant upper word | (address >> 4) in the lower word
@@ -409,9 +410,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else {
-        // ------------------------------------------------------------- epilogue (warps 5..20)
+        // ------------------------------------------------------------- epilogue (warps 8..23)
         const int q = warp & 3;         // this warp's quarter of tensor memory
-        const int wg = (warp - 1 - kMmaWarps) >> 2;  // epilogue warpgroup
+        const int wg = (warp - kProdWarps - kMmaWarps) >> 2;  // epilogue warpgroup
         const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
         const int c_begin = p.split_cols ? wg * c_span : 0;
         const int c_end = c_begin + c_span;
@@ -429,7 +430,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             {
                 TRACE_T0();
                 ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
-                if (threadIdx.x == 32 * (1 + kMmaWarps)) TRACE_ADD(3);
+                if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(3);
             }
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -464,7 +465,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     TRACE_T0();
                     tmem_ld16(taddr + c0, acc);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (threadIdx.x == 32 * (1 + kMmaWarps)) TRACE_ADD(7);
+                    if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(7);
                 }
                 if (c0 + 16 >= c_end) {
                     // all of this warp's reads of the stage are done: hand it back to the MMA warp
@@ -501,8 +502,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 
 #ifdef ACCERL_TC_TRACE
-    if (lane == 0 && (warp == 0 || warp == 1 || warp == 1 + kMmaWarps))
-        atomicAdd((unsigned long long *)(p.status + 16) + p.trace_slot * 8 + 4 + (warp > 1 ? 2 : warp),
+    if (lane == 0 && (warp == 0 || warp == kProdWarps || warp == kProdWarps + kMmaWarps))
+        atomicAdd((unsigned long long *)(p.status + 16) + p.trace_slot * 8 + 4 + (warp == 0 ? 0 : (warp == kProdWarps ? 1 : 2)),
                   (unsigned long long)(clock64() - trace_start));
 #endif
     // ---------------------------------------------------------------- teardown
@@ -512,7 +513,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kProdWarps) {
         __syncwarp();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
