@@ -210,12 +210,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int a_chunk_bytes = kTileM * CH;
     const int b_tile_bytes = p.n_tile * CH;
     // shifted mode: a stage is one box of a_rows rows that all taps of the tile read at row offsets
-    const int stage_bytes = p.shifted ? ((p.a_rows * CH + 1023) & ~1023)
+    // sub > 1 (shifted mode only): a pipeline step covers `sub` consecutive 128-row tiles, one TMA
+    // box and one accumulator each, so that the barrier round trips are paid once per step
+    const int SUB = p.sub;
+    const int box_bytes = (p.a_rows * CH + 1023) & ~1023;
+    const int stage_bytes = p.shifted ? SUB * box_bytes
                                       : p.group * (a_chunk_bytes + (RESIDENT_B ? 0 : b_tile_bytes));
     uint8_t *resident_b = smem;
     uint8_t *stages = smem + (RESIDENT_B ? ((p.n_chunks * b_tile_bytes + 1023) & ~1023) : 0);
     const int n_stages = p.n_stages, n_acc = p.n_acc_stages;
-    const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;  // column stride of an accumulator stage
+    const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;  // columns of one accumulator
+    const int acc_stride = SUB * acc_cols;               // column stride of an accumulator stage
     volatile int *abort_flag = &bars.abort_flag;
 
     {
@@ -256,7 +261,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = bars.tmem_base;
 
-    const int total_tiles = p.m_tiles * p.n_tiles;
+    const int total_tiles = ((p.m_tiles + SUB - 1) / SUB) * p.n_tiles;  // pipeline steps
 #ifdef ACCERL_TC_TRACE
     const long long trace_start = clock64();
 #endif
@@ -301,7 +306,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 mt = t / p.n_tiles;
                 nt = t - mt * p.n_tiles;
             }
-            const int row0 = mt * kTileM, brow0 = nt * p.n_tile;
+            const int row0 = mt * kTileM * SUB, brow0 = nt * p.n_tile;
             for (int gi = 0; gi < n_groups; ++gi) {
                 const int j = gi * G;
                 int sl = base_slot + gi;
@@ -322,8 +327,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t st = stages_addr + (uint32_t)s * stage_bytes;
                 if (p.shifted) {
                     if (elect_one()) {
-                        mbar_expect_tx(full, (uint32_t)(p.a_rows * CH));
-                        tma_load_2d(st, &map_a, 0, row0, full);
+                        mbar_expect_tx(full, (uint32_t)(SUB * p.a_rows * CH));
+                        for (int sub = 0; sub < SUB; ++sub)
+                            tma_load_2d(st + sub * box_bytes, &map_a, 0, row0 + sub * kTileM, full);
                     }
                 } else if (elect_one()) {
                     mbar_expect_tx(full, (uint32_t)stage_bytes);
@@ -367,7 +373,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_cols);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_stride);
             for (int gi = 0; gi < n_groups; ++gi) {
                 int sl = base_slot + gi;
                 uint32_t par = base_phase;
@@ -387,10 +393,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint32_t st_lo = ((stages_addr + (uint32_t)s * stage_bytes) >> 4) | desc_lo_flags;
                 if (elect_one()) {
                     const int t0 = j * k_steps, t1 = t0 + G * k_steps;
-                    for (int t = t0; t < t1; ++t) {
-                        const uint2 rel = s_desc[t];
-                        const uint32_t b_lo = RESIDENT_B ? rel.y : st_lo + rel.y;
-                        mma_i8(d_tmem, desc_hi | (st_lo + rel.x), desc_hi | b_lo, idesc, (uint32_t)t);
+                    for (int sub = 0; sub < SUB; ++sub) {
+                        const uint32_t sub_lo = st_lo + (uint32_t)((sub * box_bytes) >> 4);
+                        for (int t = t0; t < t1; ++t) {
+                            const uint2 rel = s_desc[t];
+                            const uint32_t b_lo = RESIDENT_B ? rel.y : st_lo + rel.y;
+                            mma_i8(d_tmem + sub * acc_cols, desc_hi | (sub_lo + rel.x), desc_hi | b_lo,
+                                   idesc, (uint32_t)t);
+                        }
                     }
                     mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
                 }
@@ -435,7 +445,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int m = mt * kTileM + q * 32 + lane;
+            for (int sub = 0; sub < SUB; ++sub) {
+            const int m = (mt * SUB + sub) * kTileM + q * 32 + lane;
             // which output position is this GEMM row?  Division-free: a float estimate of
             // m / rows_per_image corrected by stepping, a 16.16 reciprocal for the row inside the image
             // (exact for r < 65536), shifts for the power-of-two space-to-depth factor.
@@ -458,7 +469,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int8_t *dst = p.out + out_row * p.out_pitch +
                           ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
             float *ldst = p.logits_mode ? p.logits + (long long)m * p.n_actions : nullptr;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * acc_cols);
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) +
+                                   (uint32_t)(a * acc_stride + sub * acc_cols);
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 int acc[16];
                 {
@@ -467,7 +479,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                     if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(7);
                 }
-                if (c0 + 16 >= c_end) {
+                if (c0 + 16 >= c_end && sub == SUB - 1) {
                     // all of this warp's reads of the stage are done: hand it back to the MMA warp
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
@@ -498,6 +510,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
+            }  // sub
         }
     }
 
@@ -574,7 +587,7 @@ size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
 {
     const int a_chunk = kTileM * p.chunk_bytes, b_tile = p.n_tile * p.chunk_bytes;
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
-    const size_t stage = p.shifted ? (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
+    const size_t stage = p.shifted ? p.sub * (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
                                    : (size_t)p.group * (a_chunk + (resident_b ? 0 : b_tile));
     return 1024 + res + (size_t)p.n_stages * stage;
 }
@@ -595,21 +608,26 @@ bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
     p.group = 1;
     for (int g = 1; g <= p.n_chunks; ++g)
         if (p.n_chunks % g == 0 && g * per_chunk <= 16 * 1024) p.group = g;
-    {
-        const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
-        p.n_acc_stages = pow2_floor(std::min(kTcMaxAccStages, 512 / acc_cols));
+    const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
+    // Tiles per pipeline step (shifted mode): as many as still leave two accumulator stages and
+    // two shared-memory stages to each issuing warp; otherwise one.
+    for (int sub = p.shifted ? p.max_sub : 1; sub >= 1; sub /= 2) {
+        p.sub = sub;
+        p.n_acc_stages = pow2_floor(std::min(kTcMaxAccStages, 512 / (sub * acc_cols)));
+        if (p.n_acc_stages < 1) continue;
         p.n_mma = std::min(kMmaWarps, p.n_acc_stages);
-    }
-    for (int s = kTcMaxStages / p.n_mma * p.n_mma; s >= p.n_mma && s >= 2; s -= p.n_mma) {
-        p.n_stages = s;
-        if (tc_smem_bytes(p, resident_b) <= limit) {
-            const int acc_cols = p.n_tile < 32 ? 32 : p.n_tile;
-            p.n_acc_stages = pow2_floor(std::min(kTcMaxAccStages, 512 / acc_cols));
-            int cols = 32;
-            while (cols < p.n_acc_stages * acc_cols) cols *= 2;
-            p.tmem_cols = cols;
-            p.n_acc_log2 = p.n_acc_stages == 8 ? 3 : (p.n_acc_stages == 4 ? 2 : (p.n_acc_stages == 2 ? 1 : 0));
-            return true;
+        const int want = sub > 1 ? 2 * p.n_mma : std::max(2, p.n_mma);
+        if (sub > 1 && p.n_acc_stages < 2 * p.n_mma) continue;
+        for (int s = kTcMaxStages / p.n_mma * p.n_mma; s >= want; s -= p.n_mma) {
+            p.n_stages = s;
+            if (tc_smem_bytes(p, resident_b) <= limit) {
+                int cols = 32;
+                while (cols < p.n_acc_stages * sub * acc_cols) cols *= 2;
+                p.tmem_cols = cols;
+                p.n_acc_log2 = 0;
+                while ((1 << p.n_acc_log2) < p.n_acc_stages) ++p.n_acc_log2;
+                return true;
+            }
         }
     }
     return false;
@@ -619,7 +637,7 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
                       int sm_count, cudaStream_t st)
 {
     const size_t smem = tc_smem_bytes(p, resident_b);
-    const int tiles = p.m_tiles * p.n_tiles;
+    const int tiles = ((p.m_tiles + p.sub - 1) / p.sub) * p.n_tiles;
     const int grid = tiles < sm_count ? tiles : sm_count;
     cudaError_t e;
     if (resident_b) {

@@ -25,6 +25,7 @@ struct TcGemmParams {
     // shifted = 1: every chunk reads the same columns at a different row offset, so one TMA box of
     // a_rows = 128 + max(row_off) rows per tile serves all of them (needs resident weights)
     int shifted, a_rows;
+    int sub, max_sub;  // 128-row tiles per pipeline step (chosen up to max_sub in shifted mode)
     // GEMM row -> output position: row = n * rows_per_image + Y * grid_w + X, kept when
     // Y < out_h and X < out_w; stored at row n * out_rows_per_image + (Y/s) * out_grid_w + X/s,
     // byte ((Y%s) * s + X%s) * n_total + channel, rows `out_pitch` bytes apart (s = out_s2d)

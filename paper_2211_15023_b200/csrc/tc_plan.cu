@@ -271,6 +271,8 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         TcStep ts;
         memset(&ts.prm, 0, sizeof(ts.prm));
         TcGemmParams &g = ts.prm;
+        g.sub = 1;
+        g.max_sub = 1;
         const bool logits = (d.flags & ACCERL_LOGITS) != 0;
         const int n_total = round_up(d.out_c, 16);
         g.n_total = n_total;
@@ -288,6 +290,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             g.rows_per_image = Hs * Ws;
             g.grid_w = Ws;
             g.shifted = 1;
+            g.max_sub = 4;
             g.a_rows = round_up(128 + (t - 1) * Ws + (t - 1), 8);
             packed.assign((size_t)g.n_chunks * n_total * CH, 0);
             for (int by = 0; by < t; ++by)
