@@ -293,6 +293,10 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             ACCERL_CUDA_TRY(tc_launch(t.map_a, t.map_b, prm, t.resident_b, p->sm_count, st));
             break;
         }
+        case Step::MLP_FUSED:
+            ACCERL_CUDA_TRY(launch_mlp_fused(p, (const float *)obs_dev, uniforms_dev, B, logits_dev,
+                                             actions_dev, logp_dev, st));
+            break;
         case Step::SAMPLE:
             ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev,
                                           logp_dev, st));
@@ -550,6 +554,9 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
     if (!(flags & ACCERL_FLAG_FORCE_GENERIC)) {
         bool used = false;
         if ((st = build_tc_plan(p, layers, n_layers, &used)) != ACCERL_OK) return fail(st);
+        if (!used && !(flags & ACCERL_FLAG_KEEP_ACTIVATIONS) &&
+            (st = build_mlp_plan(p, layers, n_layers, &used)) != ACCERL_OK)
+            return fail(st);
     }
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <memory>
 #include <string>
 #include <vector>
 
@@ -49,7 +50,7 @@ struct LayerPlan {
 // One kernel launch of the plan: which kernel, and which part of the path it covers
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
-    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM } kind;
+    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED } kind;
     int layer = -1;
     int tc = -1;  // index into accerl_policy::tc_steps for TC_GEMM
     std::string kernel, covers;
@@ -63,6 +64,8 @@ struct TcStep {
     TcGemmParams prm;
     bool resident_b = false;
 };
+
+struct MlpFusedParams;  // mlp_fused.cu
 
 struct DeviceBuf {
     int8_t *ptr = nullptr;
@@ -82,6 +85,7 @@ struct accerl_policy {
     std::vector<accerl::LayerPlan> layers;
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
     std::vector<accerl::TcStep> tc_steps;
+    std::shared_ptr<accerl::MlpFusedParams> mlp;  // set when the whole step is one fused launch
     std::vector<int> tensor_s2d;          // space-to-depth factor of tensor t at [t + 1]
     int sm_count = 0;
     std::vector<accerl::DeviceBuf> bufs;  // bufs[0] holds the quantised input
@@ -120,6 +124,11 @@ cudaError_t launch_sample(const float *logits, const float *u, int B, int A, int
 // ACCERL_OK with *used = false when it does not
 accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
                             bool *used);
+// single-launch plan for all-FC policies on vector observations (mlp_fused.cu)
+accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
+                             bool *used);
+cudaError_t launch_mlp_fused(const accerl_policy *p, const float *obs, const float *u, int B,
+                             float *logits, int32_t *actions, float *logp, cudaStream_t st);
 accerl_status upload_bytes(accerl_policy *p, const void *host, size_t bytes, void **dev);
 
 }  // namespace accerl

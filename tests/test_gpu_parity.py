@@ -75,6 +75,22 @@ def test_full_batch_sampled_states(name):
     g.close()
 
 
+@pytest.mark.parametrize("name", ["cartpole_mlp", "lunarlander_mlp"])
+def test_single_launch_mlp_plan_odd_batches(name):
+    """Vector-observation MLPs run as one fused launch; batches around the 8-row CTA granule."""
+    import paper_2211_15023_b200 as P
+    pol = calibrated(name)
+    g = P.Policy(pol, 200, flags=0)
+    info = g.info()
+    assert info["launches_per_act"] == 1 and "mlp_fused_kernel" in info["plan"]
+    for b in (1, 7, 8, 9, 160, 199):
+        obs, u = W.observations(name, b, seed=b), W.uniforms(name, b, seed=100 + b)
+        ref = oracle.forward(pol, obs, u, keep=False)
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        compare(ref, *out)
+    g.close()
+
+
 def test_act_host_matches_device_call():
     import paper_2211_15023_b200 as P
     name = "nature_cnn_b160"
