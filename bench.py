@@ -178,6 +178,21 @@ def run_reference(args) -> None:
     }))
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: the job's step time when every rank runs its own replica."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(batch_per_rank: int, world: int, ms: float) -> float:
+    """Whole-job states/s: all ranks' states over the slowest rank's time."""
+    return batch_per_rank * world / (ms * 1e-3)
+
+
 def time_workload(P, torch, name, batch, steps, warmup, n_buffers, device, dist=None, clocks=False):
     """Times `steps` act calls with CUDA events on the launching stream; returns a dict."""
     pol = W.drawn_int8_policy(name)
@@ -211,11 +226,9 @@ def time_workload(P, torch, name, batch, steps, warmup, n_buffers, device, dist=
         time.sleep(0.15)
         sampler.__exit__()
     ms = ev0.elapsed_time(ev1) / steps
+    ms = max_over_ranks(ms, dist, u.device)
     if dist is not None:
-        t = torch.tensor([ms], device=u.device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        ms = float(t.item())
     g.check()
     info = g.info()
     # per-launch device times (a second pass over the same steps with events around each launch)
@@ -269,7 +282,7 @@ def main() -> None:
     ms = r["ms"]
     g = r["policy"]
     clocks = r["clocks"]
-    value = batch * world / (ms * 1e-3)
+    value = job_value(batch, world, ms)
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies timed)
     a = g.n_actions
@@ -292,10 +305,7 @@ def main() -> None:
     ev1.record(stream)
     torch.cuda.synchronize()
     e2e_ms = ev0.elapsed_time(ev1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
     if rank != 0:
         if dist is not None:
             dist.barrier()
@@ -367,7 +377,7 @@ def main() -> None:
                          (n_buffers, in_bytes / 1e6),
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks,
-        "e2e": {"value": batch * world / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        "e2e": {"value": job_value(batch, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": in_bytes + 4 * batch,
                 "d2h_bytes_per_step": OUT_BYTES(a) * batch},
         "gpu_launches": int(len(per) * args.steps),
