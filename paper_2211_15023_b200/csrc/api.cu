@@ -293,6 +293,15 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             ACCERL_CUDA_TRY(tc_launch(t.map_a, t.map_b, prm, t.resident_b, p->sm_count, st));
             break;
         }
+        case Step::INGEST_NHWC4:
+            ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut,
+                                                   p->bufs[p->layers[0].in_buf].ptr, B,
+                                                   p->in_h * p->in_w, p->ingest_arith, p->ingest_mul,
+                                                   p->ingest_add, st));
+            break;
+        case Step::POOL_DUAL:
+            ACCERL_CUDA_TRY(launch_maxpool_dual(p->pools[s.tc], B, st));
+            break;
         case Step::MLP_FUSED:
             ACCERL_CUDA_TRY(launch_mlp_fused(p, (const float *)obs_dev, uniforms_dev, B, logits_dev,
                                              actions_dev, logp_dev, st));
@@ -554,6 +563,8 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
     if (!(flags & ACCERL_FLAG_FORCE_GENERIC)) {
         bool used = false;
         if ((st = build_tc_plan(p, layers, n_layers, &used)) != ACCERL_OK) return fail(st);
+        if (!used && (st = build_tc_mixed_plan(p, layers, n_layers, &used)) != ACCERL_OK)
+            return fail(st);
         if (!used && !(flags & ACCERL_FLAG_KEEP_ACTIVATIONS) &&
             (st = build_mlp_plan(p, layers, n_layers, &used)) != ACCERL_OK)
             return fail(st);
@@ -687,6 +698,27 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
         return ACCERL_ERR_INVALID_ARG;
     }
     DeviceGuard guard(p->device);
+    if ((size_t)(layer + 1) < p->taps.size() && p->taps[layer + 1].ptr) {
+        // the tensor is only stored with a zero border and a fixed pixel pitch
+        const TapDesc &t = p->taps[layer + 1];
+        const int Hp = H + 2 * t.border, Wp = W + 2 * t.border;
+        std::vector<int8_t> pad;
+        try {
+            pad.resize((size_t)batch * Hp * Wp * t.pitch);
+        } catch (...) {
+            set_error("read_activation: out of host memory");
+            return ACCERL_ERR_OOM;
+        }
+        ACCERL_CUDA_TRY(cudaDeviceSynchronize());
+        ACCERL_CUDA_TRY(cudaMemcpy(pad.data(), t.ptr, pad.size(), cudaMemcpyDeviceToHost));
+        for (int b = 0; b < batch; ++b)
+            for (int c = 0; c < C; ++c)
+                for (int y = 0; y < H; ++y)
+                    for (int x = 0; x < W; ++x)
+                        dst[(((size_t)b * C + c) * H + y) * W + x] =
+                            pad[(((size_t)b * Hp + y + t.border) * Wp + x + t.border) * t.pitch + c];
+        return ACCERL_OK;
+    }
     std::vector<int8_t> tmp;
     try {
         tmp.resize((size_t)batch * H * W * Cp);

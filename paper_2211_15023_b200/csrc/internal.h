@@ -50,9 +50,10 @@ struct LayerPlan {
 // One kernel launch of the plan: which kernel, and which part of the path it covers
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
-    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED } kind;
+    enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED,
+                INGEST_NHWC4, POOL_DUAL } kind;
     int layer = -1;
-    int tc = -1;  // index into accerl_policy::tc_steps for TC_GEMM
+    int tc = -1;  // index into accerl_policy::tc_steps (TC_GEMM) or ::pools (POOL_DUAL)
     std::string kernel, covers;
 };
 
@@ -66,6 +67,19 @@ struct TcStep {
 };
 
 struct MlpFusedParams;  // mlp_fused.cu
+
+// max-pool that writes a plain NHWC output and / or a padded-border one (tc_mixed_plan.cu)
+struct PoolDualParams {
+    const int8_t *in;
+    int8_t *out_plain, *out_pad;
+    int H, W, C, OH, OW, k, stride, pad_pitch, pad_relu;
+};
+
+// where the parity tap of a tensor lives when it is not in the generic plan's buffer
+struct TapDesc {
+    const int8_t *ptr = nullptr;
+    int pitch = 0, border = 0;
+};
 
 struct DeviceBuf {
     int8_t *ptr = nullptr;
@@ -85,6 +99,8 @@ struct accerl_policy {
     std::vector<accerl::LayerPlan> layers;
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
     std::vector<accerl::TcStep> tc_steps;
+    std::vector<accerl::PoolDualParams> pools;
+    std::vector<accerl::TapDesc> taps;    // per tensor (index t + 1); empty or null ptr = generic buffer
     std::shared_ptr<accerl::MlpFusedParams> mlp;  // set when the whole step is one fused launch
     std::vector<int> tensor_s2d;          // space-to-depth factor of tensor t at [t + 1]
     int sm_count = 0;
@@ -124,6 +140,12 @@ cudaError_t launch_sample(const float *logits, const float *u, int B, int A, int
 // ACCERL_OK with *used = false when it does not
 accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
                             bool *used);
+// mixed tensor-core / CUDA-core plan for residual 3x3 conv stacks (tc_mixed_plan.cu)
+accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
+                                  bool *used);
+cudaError_t launch_maxpool_dual(const PoolDualParams &q, int B, cudaStream_t st);
+cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int HW,
+                                   int arith, uint32_t mul, uint32_t add, cudaStream_t st);
 // single-launch plan for all-FC policies on vector observations (mlp_fused.cu)
 accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
                              bool *used);

@@ -197,6 +197,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ Barriers bars;
     __shared__ __align__(16) float s_ks[kTcMaxN], s_bs[kTcMaxN];
+    __shared__ int s_skip_mul[256];
+    if (p.skip)
+        for (int i = threadIdx.x; i < p.n_total && i < 256; i += blockDim.x) s_skip_mul[i] = p.skip_mul[i];
     // per (chunk, k step): low descriptor words of the A and B operands, relative to the stage
     // (B absolute when the weights are resident), so that the issue loop is a load and an add
     __shared__ uint2 s_desc[kTcMaxChunks * 4];
@@ -464,7 +467,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
             const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
             const long long out_row =
-                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh);
+                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) +
+                p.out_row_off;
+            int8_t *dst2 = p.out2 ? p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w +
+                                              X + p.out2_row_off) * p.out2_pitch
+                                  : nullptr;
+            const int8_t *skip = p.skip ? p.skip + ((long long)n * p.out_h * p.out_w + Y * p.out_w + X) *
+                                                       p.skip_pitch
+                                        : nullptr;
             const int col0 = nt * p.n_tile;
             int8_t *dst = p.out + out_row * p.out_pitch +
                           ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
@@ -486,6 +496,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (lane == 0) mbar_arrive(acc_empty0 + 8 * a);
                 }
                 if (!valid) continue;
+                if (skip) {  // residual add in the int32 domain
+                    const uint4 sv = __ldg(reinterpret_cast<const uint4 *>(skip + col0 + c0));
+                    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        acc[i] += s_skip_mul[col0 + c0 + i] * (int)(int8_t)(sw[i >> 2] >> (8 * (i & 3)));
+                }
                 float ks[16], bs[16];
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
@@ -507,7 +524,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     } else {
                         requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
                     }
-                    *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                    if (p.out_relu | p.out2_relu) {
+                        uint32_t wr[4];
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
+                            const uint32_t neg = w[g] & 0x80808080u;
+                            wr[g] = w[g] & ~(neg | (neg - (neg >> 7)));
+                        }
+                        *reinterpret_cast<uint4 *>(dst + c0) =
+                            p.out_relu ? make_uint4(wr[0], wr[1], wr[2], wr[3])
+                                       : make_uint4(w[0], w[1], w[2], w[3]);
+                        if (dst2)
+                            *reinterpret_cast<uint4 *>(dst2 + col0 + c0) =
+                                p.out2_relu ? make_uint4(wr[0], wr[1], wr[2], wr[3])
+                                            : make_uint4(w[0], w[1], w[2], w[3]);
+                    } else {
+                        *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                        if (dst2)
+                            *reinterpret_cast<uint4 *>(dst2 + col0 + c0) = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
                 }
             }
             }  // sub

@@ -32,6 +32,16 @@ struct TcGemmParams {
     int batch, rows_per_image, grid_w, out_h, out_w;
     int out_s2d, out_rows_per_image, out_grid_w, out_pitch;
     int out_s2d_log2;
+    int out_row_off;  // added to the output row (a one-pixel border of a padded consumer layout)
+    int out_relu;     // clamp the stored codes at 0 (the only reader applies ReLU to its input)
+    // optional second copy of the output in another layout: row = n * out2_rows_per_image +
+    // Y * out2_grid_w + X + out2_row_off, `out2_pitch` bytes apart, ReLU'd if out2_relu
+    int8_t *out2;
+    int out2_rows_per_image, out2_grid_w, out2_row_off, out2_pitch, out2_relu;
+    // optional residual: acc += skip_mul[c] * skip[n, Y, X, c] from a plain NHWC tensor
+    const int8_t *skip;
+    const int32_t *skip_mul;
+    int skip_pitch;
     float inv_rows_per_image;  // 1 / rows_per_image, for the division-free row decode
     unsigned grid_w_magic;     // ceil(2^32 / grid_w)
     // epilogue

@@ -1,0 +1,444 @@
+// Tensor-core plan for residual conv stacks (the IMPALA-ResNet shape): 3x3 stride-1 pad-1
+// convolutions with 16 or 32 input channels run on tc_gemm_kernel in shifted mode, the remaining
+// layers (a first conv on 4 channels, max-pools) on CUDA-core kernels.
+//
+// A tensor read by such a conv is stored with a one-pixel zero border and 32 bytes per pixel
+// ([n][H+2][W+2][32], channels 16..31 zero when the tensor has 16), so that the conv is a valid
+// 3x3 conv on the padded image: one GEMM row per padded position, taps at row offsets
+// ky * (W+2) + kx, 32-byte rows = one K step per tap.  Borders and padding channels are zeroed
+// once at create and never written.  A tensor may be kept in two forms at once (for instance the
+// input x of a residual block: plain for the skip add, padded and ReLU'd for the block's first
+// conv); producers (the conv epilogue, the pooling kernel) write both.
+#include <string.h>
+
+#include <algorithm>
+
+#include "internal.h"
+
+namespace accerl {
+
+// ---------------------------------------------------------------------------------------
+// max-pool with up to two outputs: plain NHWC and / or padded-border (optionally ReLU'd)
+// ---------------------------------------------------------------------------------------
+__global__ void maxpool_dual_kernel(const PoolDualParams q, long long total)
+{
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    const int G = q.C / 16;  // 16-byte channel groups per pixel
+    int g = (int)(idx % G);
+    long long t = idx / G;
+    int ox = (int)(t % q.OW);
+    t /= q.OW;
+    int oy = (int)(t % q.OH);
+    long long n = t / q.OH;
+    uint32_t m[4] = {0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u};
+    for (int ky = 0; ky < q.k; ++ky)
+        for (int kx = 0; kx < q.k; ++kx) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(
+                q.in + ((n * q.H + oy * q.stride + ky) * q.W + ox * q.stride + kx) * q.C + g * 16));
+            m[0] = __vmaxs4(m[0], v.x);
+            m[1] = __vmaxs4(m[1], v.y);
+            m[2] = __vmaxs4(m[2], v.z);
+            m[3] = __vmaxs4(m[3], v.w);
+        }
+    if (q.out_plain)
+        *reinterpret_cast<uint4 *>(q.out_plain + ((n * q.OH + oy) * q.OW + ox) * q.C + g * 16) =
+            make_uint4(m[0], m[1], m[2], m[3]);
+    if (q.out_pad) {
+        if (q.pad_relu) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) m[i] = __vmaxs4(m[i], 0u);
+        }
+        const long long row = (n * (q.OH + 2) + oy + 1) * (q.OW + 2) + ox + 1;
+        *reinterpret_cast<uint4 *>(q.out_pad + row * q.pad_pitch + g * 16) =
+            make_uint4(m[0], m[1], m[2], m[3]);
+    }
+}
+
+cudaError_t launch_maxpool_dual(const PoolDualParams &q, int B, cudaStream_t st)
+{
+    const long long total = (long long)B * q.OH * q.OW * (q.C / 16);
+    maxpool_dual_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(q, total);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// uint8 NCHW frames with 4 channels -> plain int8 NHWC: four pixels per thread
+// ---------------------------------------------------------------------------------------
+template <bool ARITH>
+__global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const int8_t *__restrict__ lut,
+                                       uint4 *__restrict__ out, long long total, int HW4,
+                                       uint32_t mul, uint32_t add)
+{
+    __shared__ int8_t s_lut[256];
+    if (!ARITH) {
+        for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = lut[i];
+        __syncthreads();
+    }
+    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= total) return;
+    // idx = n * HW4 + p4: pixels 4*p4 .. 4*p4+3 of image n (HW is a multiple of 4)
+    const long long n = idx / HW4;
+    const int p4 = (int)(idx - n * HW4);
+    uint32_t plane[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        plane[c] = __ldg(reinterpret_cast<const uint32_t *>(obs + (n * 4 + c) * (4LL * HW4)) + p4);
+    uint32_t w[4];
+#pragma unroll
+    for (int px = 0; px < 4; ++px) {
+        if (ARITH) {
+            uint32_t pr[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) pr[c] = ((plane[c] >> (8 * px)) & 0xff) * mul + add;
+            const uint32_t lo = __byte_perm(pr[0], pr[1], 0x0073), hi = __byte_perm(pr[2], pr[3], 0x0073);
+            w[px] = __vminu4(__byte_perm(lo, hi, 0x5410), 0x7f7f7f7fu);
+        } else {
+            uint32_t word = 0;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                word |= (uint32_t)(uint8_t)s_lut[(plane[c] >> (8 * px)) & 0xff] << (8 * c);
+            w[px] = word;
+        }
+    }
+    out[idx] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int HW,
+                                   int arith, uint32_t mul, uint32_t add, cudaStream_t st)
+{
+    const long long total = (long long)B * (HW / 4);
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    if (arith)
+        ingest_u8_nhwc4_kernel<true><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, HW / 4, mul, add);
+    else
+        ingest_u8_nhwc4_kernel<false><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, HW / 4, mul, add);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------
+// plan
+// ---------------------------------------------------------------------------------------
+namespace {
+
+enum Role { GENERIC, POOL, TCCONV, TCFC };
+
+struct Forms {  // which stored forms of a tensor its readers need
+    bool plain = false, plain_relu = false, pad = false, pad_relu = false;
+    int8_t *p_plain = nullptr, *p_plain_relu = nullptr, *p_pad = nullptr;
+    int count() const { return (plain ? 1 : 0) + (plain_relu ? 1 : 0) + ((pad || pad_relu) ? 1 : 0); }
+};
+
+bool tcconv_ok(const accerl_layer_desc &d)
+{
+    return d.kind == ACCERL_CONV2D && d.kh == 3 && d.kw == 3 && d.stride == 1 && d.pad == 1 &&
+           (d.in_c == 16 || d.in_c == 32) && d.out_c % 16 == 0 && d.out_c <= 256 &&
+           128 + 2 * (d.in_w + 2) + 2 <= 256;
+}
+
+accerl_status alloc_zeroed(accerl_policy *p, size_t bytes, int8_t **out)
+{
+    void *d = nullptr;
+    ACCERL_CUDA_TRY(cudaMalloc(&d, bytes + 4096));  // slack: TMA boxes may start before the tail
+    p->owned.push_back(d);
+    p->workspace_bytes += bytes + 4096;
+    ACCERL_CUDA_TRY(cudaMemset(d, 0, bytes + 4096));
+    *out = (int8_t *)d;
+    return ACCERL_OK;
+}
+
+}  // namespace
+
+accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
+                                  bool *used)
+{
+    *used = false;
+    if (p->in_kind != ACCERL_IN_U8_NCHW) return ACCERL_OK;
+    const bool keep = (p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) != 0;
+    // ---- roles
+    std::vector<Role> role(n_layers);
+    int n_tc = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const accerl_layer_desc &d = layers[i];
+        const LayerPlan &L = p->layers[i];
+        if (tcconv_ok(d)) {
+            role[i] = TCCONV;
+            ++n_tc;
+        } else if (d.kind == ACCERL_MAXPOOL && (d.in_c == 16 || d.in_c == 32) && d.pad == 0) {
+            role[i] = POOL;
+        } else if (d.kind == ACCERL_FC) {
+            const int K = L.in_h * L.in_w * L.in_cp;
+            const bool fits = L.in_cp == L.in_c && K % 16 == 0 && K >= 128 &&
+                              (K + 127) / 128 <= kTcMaxChunks &&
+                              ((d.flags & ACCERL_LOGITS) ? d.out_c <= 256
+                                                         : (d.out_c % 16 == 0 && d.out_c <= kTcMaxN &&
+                                                            (d.out_c <= 256 || d.out_c % 256 == 0)));
+            if (!fits) return ACCERL_OK;
+            role[i] = TCFC;
+        } else if (d.kind == ACCERL_CONV2D && d.skip_from < 0 && i == 0) {
+            role[i] = GENERIC;  // the first conv (few input channels) stays on the dp4a kernel
+        } else {
+            return ACCERL_OK;
+        }
+        if (d.skip_from >= 0 && role[i] != TCCONV) return ACCERL_OK;
+    }
+    if (n_tc == 0) return ACCERL_OK;
+    for (int i = 0; i < n_layers; ++i)
+        if ((long long)p->max_batch * (p->layers[i].in_h + 2) * (p->layers[i].in_w + 2) + 512 >= (1LL << 31))
+            return ACCERL_OK;
+
+    // ---- forms of every tensor (index t + 1; tensor -1 is the quantised input)
+    std::vector<Forms> forms(n_layers + 1);
+    forms[0].plain = true;  // the input feeds the generic first conv
+    if (role[0] != GENERIC) return ACCERL_OK;
+    for (int j = 1; j < n_layers; ++j) {
+        const accerl_layer_desc &d = layers[j];
+        Forms &f = forms[j];  // tensor j - 1
+        const bool relu_in = (d.flags & ACCERL_RELU_IN) && !(layers[j - 1].flags & ACCERL_RELU_OUT);
+        if (role[j] == GENERIC || role[j] == POOL) {
+            if (relu_in) return ACCERL_OK;
+            f.plain = true;
+        } else if (role[j] == TCCONV) {
+            (relu_in ? f.pad_relu : f.pad) = true;
+        } else {
+            (relu_in ? f.plain_relu : f.plain) = true;
+        }
+        if (d.skip_from >= 0) forms[d.skip_from + 1].plain = true;
+    }
+    for (int t = 0; t < n_layers; ++t) {
+        Forms &f = forms[t];
+        if (f.pad && f.pad_relu) return ACCERL_OK;
+        if (keep && !f.plain && !f.pad) f.plain = true;  // the parity tap needs an un-ReLU'd form
+        if (f.count() > 2) return ACCERL_OK;
+        if (t > 0 && role[t - 1] == GENERIC && (f.count() != 1 || !f.plain)) return ACCERL_OK;
+        if (t > 0 && role[t - 1] == POOL && f.plain_relu) return ACCERL_OK;
+    }
+
+    // ---- buffers: plain forms live in the generic plan's buffers, the others are new
+    accerl_status st;
+    for (int t = 0; t < n_layers; ++t) {
+        Forms &f = forms[t];
+        const int C = t == 0 ? p->in_cp : p->layers[t - 1].out_cp;
+        const int H = t == 0 ? p->in_h : p->layers[t - 1].out_h;
+        const int W = t == 0 ? p->in_w : p->layers[t - 1].out_w;
+        if (f.plain) f.p_plain = t == 0 ? p->bufs[p->layers[0].in_buf].ptr
+                                        : p->bufs[p->layers[t - 1].out_buf].ptr;
+        if (f.plain_relu &&
+            (st = alloc_zeroed(p, (size_t)p->max_batch * H * W * C, &f.p_plain_relu)) != ACCERL_OK)
+            return st;
+        if ((f.pad || f.pad_relu) &&
+            (st = alloc_zeroed(p, (size_t)p->max_batch * (H + 2) * (W + 2) * 32, &f.p_pad)) != ACCERL_OK)
+            return st;
+    }
+
+    // ---- steps
+    auto bail = [&]() {  // the generic plan stays: forget everything built so far
+        p->taps.clear();
+        p->pools.clear();
+        p->tc_steps.clear();
+        return ACCERL_OK;
+    };
+    std::vector<Step> steps;
+    p->taps.assign(n_layers + 1, TapDesc());
+    {
+        Step s0;
+        const bool fast = p->in_c == 4 && (p->in_h * p->in_w) % 4 == 0;
+        s0.kind = fast ? Step::INGEST_NHWC4 : Step::INGEST;
+        s0.kernel = fast ? "ingest_u8_nhwc4_kernel" : "ingest_u8_kernel";
+        s0.covers = "ingest";
+        steps.push_back(s0);
+    }
+    for (int i = 0; i < n_layers; ++i) {
+        const accerl_layer_desc &d = layers[i];
+        const LayerPlan &L = p->layers[i];
+        const Forms &fin = forms[i], &fout = forms[i + 1];
+        Step s;
+        s.layer = i;
+        s.covers = "layer " + std::to_string(i);
+        if (i + 1 < n_layers && !fout.plain && (fout.pad || fout.pad_relu) && !fout.pad_relu) {
+            // parity tap from the padded, un-ReLU'd form
+            p->taps[i + 1].ptr = fout.p_pad;
+            p->taps[i + 1].pitch = 32;
+            p->taps[i + 1].border = 1;
+        }
+        if (role[i] == GENERIC) {
+            s.kind = Step::CONV_GENERIC;
+            s.kernel = L.how;
+            steps.push_back(s);
+            continue;
+        }
+        if (role[i] == POOL) {
+            PoolDualParams q;
+            memset(&q, 0, sizeof(q));
+            q.in = fin.p_plain;
+            q.out_plain = fout.plain ? fout.p_plain : nullptr;
+            q.out_pad = fout.p_pad;
+            q.pad_relu = fout.pad_relu ? 1 : 0;
+            q.pad_pitch = 32;
+            q.H = L.in_h; q.W = L.in_w; q.C = L.in_c; q.OH = L.out_h; q.OW = L.out_w;
+            q.k = d.kh; q.stride = d.stride;
+            p->pools.push_back(q);
+            s.kind = Step::POOL_DUAL;
+            s.tc = (int)p->pools.size() - 1;
+            s.kernel = "maxpool_dual_kernel";
+            steps.push_back(s);
+            continue;
+        }
+        // ---- tensor-core layer
+        TcStep ts;
+        memset(&ts.prm, 0, sizeof(ts.prm));
+        TcGemmParams &g = ts.prm;
+        const bool logits = (d.flags & ACCERL_LOGITS) != 0;
+        const int n_total = round_up(d.out_c, 16);
+        g.sub = 1;
+        g.max_sub = 1;
+        g.n_total = n_total;
+        g.n_tile = n_total > 256 ? 256 : n_total;
+        g.n_tiles = n_total / g.n_tile;
+        std::vector<int8_t> packed;
+        const int8_t *a_ptr;
+        long long a_rows_total;
+        int row_bytes;
+        if (role[i] == TCCONV) {
+            const int Hp = d.in_h + 2, Wp = d.in_w + 2;
+            g.chunk_bytes = 32;
+            g.n_chunks = 9;
+            g.rows_per_image = Hp * Wp;
+            g.grid_w = Wp;
+            g.shifted = 1;
+            g.max_sub = 2;
+            g.a_rows = round_up(128 + 2 * Wp + 2, 8);
+            packed.assign((size_t)9 * n_total * 32, 0);
+            for (int ky = 0; ky < 3; ++ky)
+                for (int kx = 0; kx < 3; ++kx) {
+                    const int j = ky * 3 + kx;
+                    g.row_off[j] = ky * Wp + kx;
+                    g.col_off[j] = 0;
+                    for (int oc = 0; oc < d.out_c; ++oc)
+                        for (int c = 0; c < d.in_c; ++c)
+                            packed[((size_t)j * n_total + oc) * 32 + c] =
+                                d.w[((oc * d.in_c + c) * 3 + ky) * 3 + kx];
+                }
+            a_ptr = fin.p_pad;
+            a_rows_total = (long long)p->max_batch * Hp * Wp;
+            row_bytes = 32;
+        } else {
+            const int K = L.in_h * L.in_w * L.in_cp;
+            g.chunk_bytes = 128;
+            g.n_chunks = (K + 127) / 128;
+            g.rows_per_image = 1;
+            g.grid_w = 1;
+            packed.assign((size_t)g.n_chunks * n_total * 128, 0);
+            for (int j = 0; j < g.n_chunks; ++j) {
+                g.row_off[j] = 0;
+                g.col_off[j] = 128 * j;
+            }
+            for (int oc = 0; oc < d.out_c; ++oc)
+                for (int c = 0; c < L.in_c; ++c)
+                    for (int y = 0; y < L.in_h; ++y)
+                        for (int x = 0; x < L.in_w; ++x) {
+                            const int ki = (y * L.in_w + x) * L.in_cp + c;
+                            packed[((size_t)(ki / 128) * n_total + oc) * 128 + ki % 128] =
+                                d.w[(size_t)oc * d.in_c + (c * L.in_h + y) * L.in_w + x];
+                        }
+            const bool relu_in = (d.flags & ACCERL_RELU_IN) && !(layers[i - 1].flags & ACCERL_RELU_OUT);
+            a_ptr = relu_in ? fin.p_plain_relu : fin.p_plain;
+            a_rows_total = p->max_batch;
+            row_bytes = K;
+        }
+        g.out_h = L.out_h;
+        g.out_w = L.out_w;
+        g.out_s2d = 1;
+        g.out_s2d_log2 = 0;
+        g.inv_rows_per_image = 1.0f / (float)g.rows_per_image;
+        g.grid_w_magic = g.grid_w == 1 ? 0xffffffffu : (unsigned)(((1ULL << 32) + g.grid_w - 1) / g.grid_w);
+        // outputs: every stored form of tensor i
+        struct OutSpec {
+            int8_t *ptr;
+            int rpi, gw, off, pitch, relu;
+        } outs[2];
+        int n_out = 0;
+        if (!logits) {
+            const int H = L.out_h, W = L.out_w;
+            if (fout.plain) outs[n_out++] = OutSpec{fout.p_plain, H * W, W, 0, n_total, 0};
+            if (fout.plain_relu) outs[n_out++] = OutSpec{fout.p_plain_relu, H * W, W, 0, n_total, 1};
+            if (fout.pad || fout.pad_relu)
+                outs[n_out++] = OutSpec{fout.p_pad, (H + 2) * (W + 2), W + 2, W + 3, 32, fout.pad_relu ? 1 : 0};
+            if (n_out == 0 || n_out > 2) return bail();
+            g.out = outs[0].ptr;
+            g.out_rows_per_image = outs[0].rpi;
+            g.out_grid_w = outs[0].gw;
+            g.out_row_off = outs[0].off;
+            g.out_pitch = outs[0].pitch;
+            g.out_relu = outs[0].relu;
+            if (n_out == 2) {
+                g.out2 = outs[1].ptr;
+                g.out2_rows_per_image = outs[1].rpi;
+                g.out2_grid_w = outs[1].gw;
+                g.out2_row_off = outs[1].off;
+                g.out2_pitch = outs[1].pitch;
+                g.out2_relu = outs[1].relu;
+            }
+        }
+        if (d.skip_from >= 0) {
+            g.skip = forms[d.skip_from + 1].p_plain;
+            g.skip_mul = L.skip_mul;
+            g.skip_pitch = p->layers[d.skip_from].out_cp;
+        }
+        g.kscale = L.kscale;
+        g.bias = L.bias;
+        g.s_out = L.s_out;
+        g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
+        {
+            volatile float inv = 1.0f / L.s_out;
+            g.inv_s_out = inv;
+        }
+        if (!logits) {
+            float kmax = 0.f, bmax = 0.f;
+            for (int c = 0; c < d.out_c; ++c) {
+                kmax = std::max(kmax, d.s_in * d.s_w[c]);
+                bmax = std::max(bmax, fabsf(d.bias[c]));
+            }
+            bool ok = false;
+            st = verify_fastdiv(g.s_out, g.inv_s_out, g.relu_out != 0, 2147483648.0f * kmax + bmax, &ok);
+            if (st != ACCERL_OK) return st;
+            g.fast_div = ok ? 1 : 0;
+        }
+        g.split_cols = g.n_tile >= 128 ? 1 : 0;
+        g.logits_mode = logits ? 1 : 0;
+        g.n_actions = p->n_actions;
+        g.status = p->status_word;
+        g.trace_slot = (int)p->tc_steps.size() % 8;
+        ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * g.chunk_bytes <= 96 * 1024;
+        if (g.shifted && !ts.resident_b) return bail();
+        if (!tc_choose_pipeline(g, ts.resident_b)) {
+            if (g.shifted) return bail();
+            ts.resident_b = false;
+            if (!tc_choose_pipeline(g, false)) return bail();
+        }
+        void *w_dev = nullptr;
+        if ((st = upload_bytes(p, packed.data(), packed.size(), &w_dev)) != ACCERL_OK) return st;
+        if ((st = tc_make_map(ts.map_a, a_ptr, a_rows_total, row_bytes, row_bytes,
+                              g.shifted ? g.a_rows : 128, g.chunk_bytes)) != ACCERL_OK)
+            return st;
+        if ((st = tc_make_map(ts.map_b, w_dev, (long long)g.n_chunks * n_total, g.chunk_bytes,
+                              g.chunk_bytes, g.n_tile, g.chunk_bytes)) != ACCERL_OK)
+            return st;
+        p->tc_steps.push_back(ts);
+        s.kind = Step::TC_GEMM;
+        s.tc = (int)p->tc_steps.size() - 1;
+        s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
+        if (g.fast_div) s.kernel += "[3-step divide verified]";
+        steps.push_back(s);
+    }
+    Step ss;
+    ss.kind = Step::SAMPLE;
+    ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
+    ss.covers = "sample";
+    steps.push_back(ss);
+    p->steps = steps;
+    *used = true;
+    return ACCERL_OK;
+}
+
+}  // namespace accerl
