@@ -295,9 +295,14 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
         }
         case Step::INGEST_NHWC4:
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut,
-                                                   p->bufs[p->layers[0].in_buf].ptr, B,
-                                                   p->in_h * p->in_w, p->ingest_arith, p->ingest_mul,
-                                                   p->ingest_add, st));
+                                                   p->bufs[p->layers[0].in_buf].ptr, B, p->in_h,
+                                                   p->in_w, p->in_h, p->in_w, 0, 0, p->ingest_arith,
+                                                   p->ingest_mul, p->ingest_add, st));
+            break;
+        case Step::INGEST_PAD4:
+            ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut, p->in_pad4, B,
+                                                   p->in_h, p->in_w, p->in_h + 2, p->in_pad4_w, 1, 4,
+                                                   p->ingest_arith, p->ingest_mul, p->ingest_add, st));
             break;
         case Step::POOL_DUAL:
             ACCERL_CUDA_TRY(launch_maxpool_dual(p->pools[s.tc], B, st));
@@ -701,10 +706,9 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
     if ((size_t)(layer + 1) < p->taps.size() && p->taps[layer + 1].ptr) {
         // the tensor is only stored with a zero border and a fixed pixel pitch
         const TapDesc &t = p->taps[layer + 1];
-        const int Hp = H + 2 * t.border, Wp = W + 2 * t.border;
         std::vector<int8_t> pad;
         try {
-            pad.resize((size_t)batch * Hp * Wp * t.pitch);
+            pad.resize((size_t)batch * t.hpitch * t.wpitch * t.pitch);
         } catch (...) {
             set_error("read_activation: out of host memory");
             return ACCERL_ERR_OOM;
@@ -716,7 +720,7 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
                 for (int y = 0; y < H; ++y)
                     for (int x = 0; x < W; ++x)
                         dst[(((size_t)b * C + c) * H + y) * W + x] =
-                            pad[(((size_t)b * Hp + y + t.border) * Wp + x + t.border) * t.pitch + c];
+                            pad[(((size_t)b * t.hpitch + y + t.off_y) * t.wpitch + x + t.off_x) * t.pitch + c];
         return ACCERL_OK;
     }
     std::vector<int8_t> tmp;

@@ -51,7 +51,7 @@ struct LayerPlan {
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
     enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED,
-                INGEST_NHWC4, POOL_DUAL } kind;
+                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4 } kind;
     int layer = -1;
     int tc = -1;  // index into accerl_policy::tc_steps (TC_GEMM) or ::pools (POOL_DUAL)
     std::string kernel, covers;
@@ -73,12 +73,15 @@ struct PoolDualParams {
     const int8_t *in;
     int8_t *out_plain, *out_pad;
     int H, W, C, OH, OW, k, stride, pad_pitch, pad_relu;
+    int in_wpitch;  // pixels per stored input row (>= W)
 };
 
 // where the parity tap of a tensor lives when it is not in the generic plan's buffer
 struct TapDesc {
     const int8_t *ptr = nullptr;
-    int pitch = 0, border = 0;
+    int pitch = 0;               // bytes per stored pixel
+    int hpitch = 0, wpitch = 0;  // stored rows per image, pixels per stored row
+    int off_y = 0, off_x = 0;    // where pixel (0, 0) sits
 };
 
 struct DeviceBuf {
@@ -100,6 +103,8 @@ struct accerl_policy {
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
     std::vector<accerl::TcStep> tc_steps;
     std::vector<accerl::PoolDualParams> pools;
+    int8_t *in_pad4 = nullptr;            // frames as [n][H+2][PW][4] with the image at (1, 4)
+    int in_pad4_w = 0;
     std::vector<accerl::TapDesc> taps;    // per tensor (index t + 1); empty or null ptr = generic buffer
     std::shared_ptr<accerl::MlpFusedParams> mlp;  // set when the whole step is one fused launch
     std::vector<int> tensor_s2d;          // space-to-depth factor of tensor t at [t + 1]
@@ -144,8 +149,9 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
 accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
                                   bool *used);
 cudaError_t launch_maxpool_dual(const PoolDualParams &q, int B, cudaStream_t st);
-cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int HW,
-                                   int arith, uint32_t mul, uint32_t add, cudaStream_t st);
+cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int H, int W,
+                                   int out_hpitch, int out_wpitch, int off_y, int off_x, int arith,
+                                   uint32_t mul, uint32_t add, cudaStream_t st);
 // single-launch plan for all-FC policies on vector observations (mlp_fused.cu)
 accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
                              bool *used);

@@ -35,7 +35,7 @@ __global__ void maxpool_dual_kernel(const PoolDualParams q, long long total)
     for (int ky = 0; ky < q.k; ++ky)
         for (int kx = 0; kx < q.k; ++kx) {
             const uint4 v = __ldg(reinterpret_cast<const uint4 *>(
-                q.in + ((n * q.H + oy * q.stride + ky) * q.W + ox * q.stride + kx) * q.C + g * 16));
+                q.in + ((n * q.H + oy * q.stride + ky) * q.in_wpitch + ox * q.stride + kx) * q.C + g * 16));
             m[0] = __vmaxs4(m[0], v.x);
             m[1] = __vmaxs4(m[1], v.y);
             m[2] = __vmaxs4(m[2], v.z);
@@ -67,7 +67,8 @@ cudaError_t launch_maxpool_dual(const PoolDualParams &q, int B, cudaStream_t st)
 // ---------------------------------------------------------------------------------------
 template <bool ARITH>
 __global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const int8_t *__restrict__ lut,
-                                       uint4 *__restrict__ out, long long total, int HW4,
+                                       int8_t *__restrict__ out, long long total, int H, int W4,
+                                       int out_hpitch, int out_wpitch, int off_y, int off_x,
                                        uint32_t mul, uint32_t add)
 {
     __shared__ int8_t s_lut[256];
@@ -77,13 +78,16 @@ __global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const in
     }
     long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= total) return;
-    // idx = n * HW4 + p4: pixels 4*p4 .. 4*p4+3 of image n (HW is a multiple of 4)
-    const long long n = idx / HW4;
-    const int p4 = (int)(idx - n * HW4);
+    // idx = (n * H + y) * W4 + x4: pixels 4*x4 .. 4*x4+3 of row y of image n (W is a multiple of 4)
+    const int x4 = (int)(idx % W4);
+    long long t = idx / W4;
+    const int y = (int)(t % H);
+    const long long n = t / H;
+    const int W = 4 * W4;
     uint32_t plane[4];
 #pragma unroll
     for (int c = 0; c < 4; ++c)
-        plane[c] = __ldg(reinterpret_cast<const uint32_t *>(obs + (n * 4 + c) * (4LL * HW4)) + p4);
+        plane[c] = __ldg(reinterpret_cast<const uint32_t *>(obs + ((n * 4 + c) * H + y) * W) + x4);
     uint32_t w[4];
 #pragma unroll
     for (int px = 0; px < 4; ++px) {
@@ -101,18 +105,23 @@ __global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const in
             w[px] = word;
         }
     }
-    out[idx] = make_uint4(w[0], w[1], w[2], w[3]);
+    // off_x is a multiple of 4 pixels, so the 16-byte store stays aligned
+    *reinterpret_cast<uint4 *>(out + (((n * out_hpitch + y + off_y) * out_wpitch) + 4 * x4 + off_x) * 4LL) =
+        make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int HW,
-                                   int arith, uint32_t mul, uint32_t add, cudaStream_t st)
+cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int H, int W,
+                                   int out_hpitch, int out_wpitch, int off_y, int off_x, int arith,
+                                   uint32_t mul, uint32_t add, cudaStream_t st)
 {
-    const long long total = (long long)B * (HW / 4);
+    const long long total = (long long)B * H * (W / 4);
     const unsigned blocks = (unsigned)((total + 255) / 256);
     if (arith)
-        ingest_u8_nhwc4_kernel<true><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, HW / 4, mul, add);
+        ingest_u8_nhwc4_kernel<true><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
+                                                            out_wpitch, off_y, off_x, mul, add);
     else
-        ingest_u8_nhwc4_kernel<false><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, HW / 4, mul, add);
+        ingest_u8_nhwc4_kernel<false><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
+                                                             out_wpitch, off_y, off_x, mul, add);
     return cudaGetLastError();
 }
 
@@ -121,7 +130,7 @@ cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t
 // ---------------------------------------------------------------------------------------
 namespace {
 
-enum Role { GENERIC, POOL, TCCONV, TCFC };
+enum Role { GENERIC, POOL, TCCONV, TCFC, TCFIRST };
 
 struct Forms {  // which stored forms of a tensor its readers need
     bool plain = false, plain_relu = false, pad = false, pad_relu = false;
@@ -176,7 +185,12 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             if (!fits) return ACCERL_OK;
             role[i] = TCFC;
         } else if (d.kind == ACCERL_CONV2D && d.skip_from < 0 && i == 0) {
-            role[i] = GENERIC;  // the first conv (few input channels) stays on the dp4a kernel
+            // A first conv on 4-channel frames: tensor cores if its only reader is a max-pool (see
+            // the TCFIRST branch below), else the dp4a kernel.
+            const bool toeplitz = d.in_c == 4 && d.kh == 3 && d.kw == 3 && d.stride == 1 && d.pad == 1 &&
+                                  (d.out_c == 16 || d.out_c == 32) && d.in_w % 4 == 0 && n_layers > 1 &&
+                                  layers[1].kind == ACCERL_MAXPOOL && !(d.flags & ACCERL_RELU_IN);
+            role[i] = toeplitz ? TCFIRST : GENERIC;
         } else {
             return ACCERL_OK;
         }
@@ -190,7 +204,9 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
     // ---- forms of every tensor (index t + 1; tensor -1 is the quantised input)
     std::vector<Forms> forms(n_layers + 1);
     forms[0].plain = true;  // the input feeds the generic first conv
-    if (role[0] != GENERIC) return ACCERL_OK;
+    if (role[0] != GENERIC && role[0] != TCFIRST) return ACCERL_OK;
+    for (int j = 1; j < n_layers; ++j)
+        if (layers[j].skip_from == 0 && role[0] == TCFIRST) role[0] = GENERIC;  // tensor 0 must be pool-only
     for (int j = 1; j < n_layers; ++j) {
         const accerl_layer_desc &d = layers[j];
         Forms &f = forms[j];  // tensor j - 1
@@ -210,7 +226,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if (f.pad && f.pad_relu) return ACCERL_OK;
         if (keep && !f.plain && !f.pad) f.plain = true;  // the parity tap needs an un-ReLU'd form
         if (f.count() > 2) return ACCERL_OK;
-        if (t > 0 && role[t - 1] == GENERIC && (f.count() != 1 || !f.plain)) return ACCERL_OK;
+        if (t > 0 && (role[t - 1] == GENERIC || role[t - 1] == TCFIRST) && (f.count() != 1 || !f.plain))
+            return ACCERL_OK;
         if (t > 0 && role[t - 1] == POOL && f.plain_relu) return ACCERL_OK;
     }
 
@@ -231,6 +248,21 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             return st;
     }
 
+    // ---- first conv on tensor cores: frames stored as [n][H+2][PW][4 B] with the image at row 1,
+    // pixel 4, PW a multiple of 8 pixels, so that 8 pixels form one 32-byte GEMM row; its output is
+    // plain NHWC with rows of OW8 * 8 pixels
+    const int W0 = p->in_w, H0 = p->in_h;
+    const int PW = round_up(4 + W0 + 1, 8), PW8 = PW / 8, OW8 = (W0 + 7) / 8;
+    int8_t *first_out = nullptr;
+    if (role[0] == TCFIRST) {
+        if ((st = alloc_zeroed(p, (size_t)p->max_batch * (H0 + 2) * PW * 4, &p->in_pad4)) != ACCERL_OK)
+            return st;
+        p->in_pad4_w = PW;
+        if ((st = alloc_zeroed(p, (size_t)p->max_batch * H0 * OW8 * 8 * layers[0].out_c, &first_out)) !=
+            ACCERL_OK)
+            return st;
+    }
+
     // ---- steps
     auto bail = [&]() {  // the generic plan stays: forget everything built so far
         p->taps.clear();
@@ -242,9 +274,18 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
     p->taps.assign(n_layers + 1, TapDesc());
     {
         Step s0;
-        const bool fast = p->in_c == 4 && (p->in_h * p->in_w) % 4 == 0;
-        s0.kind = fast ? Step::INGEST_NHWC4 : Step::INGEST;
+        const bool fast = p->in_c == 4 && p->in_w % 4 == 0;
+        s0.kind = role[0] == TCFIRST ? Step::INGEST_PAD4 : (fast ? Step::INGEST_NHWC4 : Step::INGEST);
         s0.kernel = fast ? "ingest_u8_nhwc4_kernel" : "ingest_u8_kernel";
+        if (role[0] == TCFIRST) {
+            TapDesc &td = p->taps[0];
+            td.ptr = p->in_pad4;
+            td.pitch = 4;
+            td.hpitch = H0 + 2;
+            td.wpitch = PW;
+            td.off_y = 1;
+            td.off_x = 4;
+        }
         s0.covers = "ingest";
         steps.push_back(s0);
     }
@@ -257,9 +298,12 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         s.covers = "layer " + std::to_string(i);
         if (i + 1 < n_layers && !fout.plain && (fout.pad || fout.pad_relu) && !fout.pad_relu) {
             // parity tap from the padded, un-ReLU'd form
-            p->taps[i + 1].ptr = fout.p_pad;
-            p->taps[i + 1].pitch = 32;
-            p->taps[i + 1].border = 1;
+            TapDesc &td = p->taps[i + 1];
+            td.ptr = fout.p_pad;
+            td.pitch = 32;
+            td.hpitch = L.out_h + 2;
+            td.wpitch = L.out_w + 2;
+            td.off_y = td.off_x = 1;
         }
         if (role[i] == GENERIC) {
             s.kind = Step::CONV_GENERIC;
@@ -270,7 +314,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if (role[i] == POOL) {
             PoolDualParams q;
             memset(&q, 0, sizeof(q));
-            q.in = fin.p_plain;
+            q.in = (i == 1 && role[0] == TCFIRST) ? first_out : fin.p_plain;
+            q.in_wpitch = (i == 1 && role[0] == TCFIRST) ? OW8 * 8 : L.in_w;
             q.out_plain = fout.plain ? fout.p_plain : nullptr;
             q.out_pad = fout.p_pad;
             q.pad_relu = fout.pad_relu ? 1 : 0;
@@ -289,7 +334,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         memset(&ts.prm, 0, sizeof(ts.prm));
         TcGemmParams &g = ts.prm;
         const bool logits = (d.flags & ACCERL_LOGITS) != 0;
-        const int n_total = round_up(d.out_c, 16);
+        const int n_total = role[i] == TCFIRST ? 8 * d.out_c : round_up(d.out_c, 16);
         g.sub = 1;
         g.max_sub = 1;
         g.n_total = n_total;
@@ -299,7 +344,50 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         const int8_t *a_ptr;
         long long a_rows_total;
         int row_bytes;
-        if (role[i] == TCCONV) {
+        const float *ks_dev = L.kscale, *bs_dev = L.bias;
+        if (role[i] == TCFIRST) {
+            // GEMM row = 8 consecutive padded pixels (32 B); output column j * out_c + oc is output
+            // pixel j of the group.  Input pixel (row ky, offset d8 * 8 + pin from the group's
+            // first pixel) meets tap kx = d8 * 8 + pin - j - 3 of output pixel j.
+            g.chunk_bytes = 32;
+            g.n_chunks = 6;
+            g.rows_per_image = (H0 + 2) * PW8;
+            g.grid_w = PW8;
+            g.shifted = 1;
+            g.a_rows = round_up(128 + 2 * PW8 + 1, 8);
+            packed.assign((size_t)6 * n_total * 32, 0);
+            for (int ky = 0; ky < 3; ++ky)
+                for (int d8 = 0; d8 < 2; ++d8) {
+                    const int j = ky * 2 + d8;
+                    g.row_off[j] = ky * PW8 + d8;
+                    g.col_off[j] = 0;
+                    for (int px = 0; px < 8; ++px)
+                        for (int oc = 0; oc < d.out_c; ++oc)
+                            for (int pin = 0; pin < 8; ++pin) {
+                                const int kx = d8 * 8 + pin - px - 3;
+                                if (kx < 0 || kx > 2) continue;
+                                for (int c = 0; c < 4; ++c)
+                                    packed[((size_t)j * n_total + px * d.out_c + oc) * 32 + pin * 4 + c] =
+                                        d.w[((oc * 4 + c) * 3 + ky) * 3 + kx];
+                            }
+                }
+            a_ptr = p->in_pad4;
+            a_rows_total = (long long)p->max_batch * (H0 + 2) * PW8;
+            row_bytes = 32;
+            // per-column scales: the channel's, repeated for the 8 pixels
+            std::vector<float> ks(n_total), bs(n_total);
+            for (int px = 0; px < 8; ++px)
+                for (int oc = 0; oc < d.out_c; ++oc) {
+                    volatile float k = d.s_in * d.s_w[oc];
+                    ks[px * d.out_c + oc] = k;
+                    bs[px * d.out_c + oc] = d.bias[oc];
+                }
+            void *kd = nullptr, *bd = nullptr;
+            if ((st = upload_bytes(p, ks.data(), ks.size() * 4, &kd)) != ACCERL_OK) return st;
+            if ((st = upload_bytes(p, bs.data(), bs.size() * 4, &bd)) != ACCERL_OK) return st;
+            ks_dev = (const float *)kd;
+            bs_dev = (const float *)bd;
+        } else if (role[i] == TCCONV) {
             const int Hp = d.in_h + 2, Wp = d.in_w + 2;
             g.chunk_bytes = 32;
             g.n_chunks = 9;
@@ -347,7 +435,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             row_bytes = K;
         }
         g.out_h = L.out_h;
-        g.out_w = L.out_w;
+        g.out_w = role[i] == TCFIRST ? OW8 : L.out_w;
         g.out_s2d = 1;
         g.out_s2d_log2 = 0;
         g.inv_rows_per_image = 1.0f / (float)g.rows_per_image;
@@ -358,12 +446,21 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             int rpi, gw, off, pitch, relu;
         } outs[2];
         int n_out = 0;
-        if (!logits) {
+        if (role[i] == TCFIRST) {
+            outs[n_out++] = OutSpec{first_out, L.out_h * OW8, OW8, 0, n_total, 0};
+            TapDesc &td = p->taps[i + 1];
+            td.ptr = first_out;
+            td.pitch = d.out_c;
+            td.hpitch = L.out_h;
+            td.wpitch = OW8 * 8;
+        } else if (!logits) {
             const int H = L.out_h, W = L.out_w;
             if (fout.plain) outs[n_out++] = OutSpec{fout.p_plain, H * W, W, 0, n_total, 0};
             if (fout.plain_relu) outs[n_out++] = OutSpec{fout.p_plain_relu, H * W, W, 0, n_total, 1};
             if (fout.pad || fout.pad_relu)
                 outs[n_out++] = OutSpec{fout.p_pad, (H + 2) * (W + 2), W + 2, W + 3, 32, fout.pad_relu ? 1 : 0};
+        }
+        if (!logits) {
             if (n_out == 0 || n_out > 2) return bail();
             g.out = outs[0].ptr;
             g.out_rows_per_image = outs[0].rpi;
@@ -385,8 +482,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             g.skip_mul = L.skip_mul;
             g.skip_pitch = p->layers[d.skip_from].out_cp;
         }
-        g.kscale = L.kscale;
-        g.bias = L.bias;
+        g.kscale = ks_dev;
+        g.bias = bs_dev;
         g.s_out = L.s_out;
         g.relu_out = (d.flags & ACCERL_RELU_OUT) != 0;
         {
