@@ -187,7 +187,9 @@ struct __align__(8) Barriers {
 
 }  // namespace
 
-template <bool RESIDENT_B>
+// EXTRAS compiles in the residual add, the second output and the stored-code ReLU; layers that
+// use none of them run the leaner instantiation (the epilogue is bound by instruction issue).
+template <bool RESIDENT_B, bool EXTRAS>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcGemmParams p)
@@ -198,7 +200,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __shared__ Barriers bars;
     __shared__ __align__(16) float s_ks[kTcMaxN], s_bs[kTcMaxN];
     __shared__ int s_skip_mul[256];
-    if (p.skip)
+    if (EXTRAS && p.skip)
         for (int i = threadIdx.x; i < p.n_total && i < 256; i += blockDim.x) s_skip_mul[i] = p.skip_mul[i];
     // per (chunk, k step): low descriptor words of the A and B operands, relative to the stage
     // (B absolute when the weights are resident), so that the issue loop is a load and an add
@@ -469,10 +471,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const long long out_row =
                 (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) +
                 p.out_row_off;
-            int8_t *dst2 = p.out2 ? p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w +
+            int8_t *dst2 = (EXTRAS && p.out2) ? p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w +
                                               X + p.out2_row_off) * p.out2_pitch
                                   : nullptr;
-            const int8_t *skip = p.skip ? p.skip + ((long long)n * p.out_h * p.out_w + Y * p.out_w + X) *
+            const int8_t *skip = (EXTRAS && p.skip) ? p.skip + ((long long)n * p.out_h * p.out_w + Y * p.out_w + X) *
                                                        p.skip_pitch
                                         : nullptr;
             const int col0 = nt * p.n_tile;
@@ -496,7 +498,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (lane == 0) mbar_arrive(acc_empty0 + 8 * a);
                 }
                 if (!valid) continue;
-                if (skip) {  // residual add in the int32 domain
+                if (EXTRAS && skip) {  // residual add in the int32 domain
                     const uint4 sv = __ldg(reinterpret_cast<const uint4 *>(skip + col0 + c0));
                     const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
@@ -524,7 +526,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     } else {
                         requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
                     }
-                    if (p.out_relu | p.out2_relu) {
+                    if (EXTRAS && (p.out_relu | p.out2_relu)) {
                         uint32_t wr[4];
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
@@ -540,7 +542,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                             : make_uint4(w[0], w[1], w[2], w[3]);
                     } else {
                         *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
-                        if (dst2)
+                        if (EXTRAS && dst2)
                             *reinterpret_cast<uint4 *>(dst2 + col0 + c0) = make_uint4(w[0], w[1], w[2], w[3]);
                     }
                 }
@@ -674,20 +676,16 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
     const size_t smem = tc_smem_bytes(p, resident_b);
     const int tiles = ((p.m_tiles + p.sub - 1) / p.sub) * p.n_tiles;
     const int grid = tiles < sm_count ? tiles : sm_count;
-    cudaError_t e;
-    if (resident_b) {
-        e = cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem);
+    const bool extras = p.skip || p.out2 || p.out_relu || p.out2_relu;
+    auto go = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        tc_gemm_kernel<true><<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a,
-                                                      *(const CUtensorMap *)map_b, p);
-    } else {
-        e = cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem);
-        if (e != cudaSuccess) return e;
-        tc_gemm_kernel<false><<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a,
-                                                       *(const CUtensorMap *)map_b, p);
-    }
+        kernel<<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, p);
+        return cudaSuccess;
+    };
+    cudaError_t e = resident_b ? (extras ? go(tc_gemm_kernel<true, true>) : go(tc_gemm_kernel<true, false>))
+                               : (extras ? go(tc_gemm_kernel<false, true>) : go(tc_gemm_kernel<false, false>));
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
