@@ -33,7 +33,7 @@ constexpr int kEpiGroups = 4;                       // epilogue warpgroups
 constexpr int kMmaWarps = 4;                        // MMA-issuing warps
 constexpr int kProdWarps = kMmaWarps;                // TMA-issuing warps, one per MMA warp's ring
 constexpr int kThreads = 32 * (kProdWarps + kMmaWarps) + 128 * kEpiGroups;
-constexpr long long kWaitLimitCycles = 4000000000LL;  // about two seconds
+constexpr int kWaitLimitPolls = 1 << 23;              // at 256 ns a poll: about two seconds
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
@@ -82,22 +82,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after kWaitLimitCycles or as soon as another role has given up.
+// Bounded wait: gives up after kWaitLimitPolls polls or as soon as another role has given up.
+// The pause between polls doubles up to 256 ns: a warp that waits for a whole tile must not take
+// issue slots from the working ones, one that waits briefly still wakes up quickly.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int *status, int code)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        __nanosleep(32);  // polling warps must not take issue slots from the working ones
+    unsigned ns = 32;
+    for (int i = 0; i < kWaitLimitPolls; ++i) {
+        __nanosleep(ns);
+        if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
-            *abort_flag = 1;
-            atomicOr(status, code);
-            return false;
-        }
+        if (ns < 256) ns <<= 1;
     }
-    return true;
+    *abort_flag = 1;
+    atomicOr(status, code);
+    return false;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,

@@ -501,7 +501,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             if (st != ACCERL_OK) return st;
             g.fast_div = ok ? 1 : 0;
         }
-        g.split_cols = g.n_tile >= 128 ? 1 : 0;
+        g.split_cols = g.n_tile > 128 ? 1 : 0;
         g.logits_mode = logits ? 1 : 0;
         g.n_actions = p->n_actions;
         g.status = p->status_word;
