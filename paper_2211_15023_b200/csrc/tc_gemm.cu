@@ -186,6 +186,152 @@ struct __align__(8) Barriers {
     int abort_flag;
 };
 
+// What the epilogue role needs from the kernel's set-up.
+struct EpiCtx {
+    uint32_t tmem_base, acc_full0, acc_empty0;
+    int total_tiles, n_acc, acc_stride, acc_cols, sub;
+    const float *s_ks, *s_bs;
+    const int *s_skip_mul;
+    volatile int *abort_flag;
+};
+
+enum { kEpiFastDiv = 0, kEpiTieCheck = 1, kEpiLogits = 2 };
+
+// Epilogue role (warps 8..23): drain accumulators, requantise, store.  The per-layer switches are
+// template parameters, chosen once per launch, so that the loop over 16-column pieces is straight
+// line code: the epilogue is bound by instruction issue.  Rows that are no output position are
+// computed like the others and only their stores are skipped, which keeps the warp converged.
+template <bool EXTRAS, int MODE, bool RELU>
+__device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
+{
+    const int q = warp & 3;         // this warp's quarter of tensor memory
+    const int wg = (warp - kProdWarps - kMmaWarps) >> 2;  // epilogue warpgroup
+    const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
+    const int c_begin = p.split_cols ? wg * c_span : 0;
+    const int c_end = c_begin + c_span;
+    const bool has_skip = EXTRAS && p.skip != nullptr, has_out2 = EXTRAS && p.out2 != nullptr;
+    const float s_out = p.s_out, inv_s_out = p.inv_s_out;
+    int tile_i = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < c.total_tiles && ok; t += gridDim.x, ++tile_i) {
+        if (!p.split_cols && (tile_i % kEpiGroups) != wg) continue;
+        int mt = t, nt = 0;
+        if (p.n_tiles != 1) {
+            mt = t / p.n_tiles;
+            nt = t - mt * p.n_tiles;
+        }
+        const int a = tile_i & (c.n_acc - 1);  // n_acc is a power of two
+        const uint32_t apar = (tile_i >> p.n_acc_log2) & 1;
+        {
+            TRACE_T0();
+            ok = mbar_wait(c.acc_full0 + 8 * a, apar, c.abort_flag, p.status, 16);
+            if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(3);
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int col0 = nt * p.n_tile;
+        for (int sub = 0; sub < c.sub; ++sub) {
+            const int m = (mt * c.sub + sub) * kTileM + q * 32 + lane;
+            // which output position is this GEMM row?  Division-free: a float estimate of
+            // m / rows_per_image corrected by stepping, a 16.16 reciprocal for the row inside the
+            // image (exact for r < 65536), shifts for the power-of-two space-to-depth factor.
+            int n = __float2int_rz(__int2float_rn(m) * p.inv_rows_per_image);
+            int r = m - n * p.rows_per_image;
+            while (r < 0) {
+                --n;
+                r += p.rows_per_image;
+            }
+            while (r >= p.rows_per_image) {
+                ++n;
+                r -= p.rows_per_image;
+            }
+            const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
+            const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
+            const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
+            const long long out_row =
+                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) +
+                p.out_row_off;
+            int8_t *dst = p.out + out_row * p.out_pitch +
+                          ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
+            int8_t *dst2 = nullptr;
+            const int8_t *skip = nullptr;
+            if (EXTRAS) {
+                if (has_out2)
+                    dst2 = p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w + X +
+                                     p.out2_row_off) * p.out2_pitch + col0;
+                if (has_skip)
+                    skip = p.skip + ((long long)n * p.out_h * p.out_w + Y * p.out_w + X) * p.skip_pitch + col0;
+            }
+            float *ldst = MODE == kEpiLogits ? p.logits + (long long)m * p.n_actions : nullptr;
+            const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) +
+                                   (uint32_t)(a * c.acc_stride + sub * c.acc_cols);
+            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+                int acc[16];
+                {
+                    TRACE_T0();
+                    tmem_ld16(taddr + c0, acc);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(7);
+                }
+                if (c0 + 16 >= c_end && sub == c.sub - 1) {
+                    // all of this warp's reads of the stage are done: hand it back to the MMA warp
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(c.acc_empty0 + 8 * a);
+                }
+                if (EXTRAS && has_skip) {  // residual add in the int32 domain
+                    uint4 sv = make_uint4(0, 0, 0, 0);
+                    if (valid) sv = __ldg(reinterpret_cast<const uint4 *>(skip + c0));
+                    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        acc[i] += c.s_skip_mul[col0 + c0 + i] * (int)(int8_t)(sw[i >> 2] >> (8 * (i & 3)));
+                }
+                float ks[16], bs[16];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    const float4 kv = *reinterpret_cast<const float4 *>(&c.s_ks[col0 + c0 + 4 * g]);
+                    const float4 bv = *reinterpret_cast<const float4 *>(&c.s_bs[col0 + c0 + 4 * g]);
+                    ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                    bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+                }
+                if (MODE == kEpiLogits) {
+                    if (valid) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (col0 + c0 + i < p.n_actions)
+                                ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
+                    }
+                    continue;
+                }
+                uint32_t w[4];
+                if (MODE == kEpiFastDiv) requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+                else requant16(acc, ks, bs, RELU, s_out, inv_s_out, w);
+                const uint4 plain = make_uint4(w[0], w[1], w[2], w[3]);
+                if (EXTRAS) {
+                    uint4 relu = plain;
+                    if (p.out_relu | p.out2_relu) {
+                        uint32_t wr[4];
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
+                            const uint32_t neg = w[g] & 0x80808080u;
+                            wr[g] = w[g] & ~(neg | (neg - (neg >> 7)));
+                        }
+                        relu = make_uint4(wr[0], wr[1], wr[2], wr[3]);
+                    }
+                    if (valid) {
+                        *reinterpret_cast<uint4 *>(dst + c0) = p.out_relu ? relu : plain;
+                        if (has_out2) *reinterpret_cast<uint4 *>(dst2 + c0) = p.out2_relu ? relu : plain;
+                    }
+                } else if (valid) {
+                    *reinterpret_cast<uint4 *>(dst + c0) = plain;
+                }
+            }
+        }
+    }
+}
+
 }  // namespace
 
 // EXTRAS compiles in the residual add, the second output and the stored-code ReLU; layers that
@@ -427,128 +573,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------------------------------------- epilogue (warps 8..23)
-        const int q = warp & 3;         // this warp's quarter of tensor memory
-        const int wg = (warp - kProdWarps - kMmaWarps) >> 2;  // epilogue warpgroup
-        const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
-        const int c_begin = p.split_cols ? wg * c_span : 0;
-        const int c_end = c_begin + c_span;
-        int tile_i = 0;
-        bool ok = true;
-        for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++tile_i) {
-            if (!p.split_cols && (tile_i % kEpiGroups) != wg) continue;
-            int mt = t, nt = 0;
-            if (p.n_tiles != 1) {
-                mt = t / p.n_tiles;
-                nt = t - mt * p.n_tiles;
-            }
-            const int a = tile_i & (n_acc - 1);  // n_acc is a power of two
-            const uint32_t apar = (tile_i >> p.n_acc_log2) & 1;
-            {
-                TRACE_T0();
-                ok = mbar_wait(smem_u32(&bars.acc_full[a]), apar, abort_flag, p.status, 16);
-                if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(3);
-            }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            for (int sub = 0; sub < SUB; ++sub) {
-            const int m = (mt * SUB + sub) * kTileM + q * 32 + lane;
-            // which output position is this GEMM row?  Division-free: a float estimate of
-            // m / rows_per_image corrected by stepping, a 16.16 reciprocal for the row inside the image
-            // (exact for r < 65536), shifts for the power-of-two space-to-depth factor.
-            int n = __float2int_rz(__int2float_rn(m) * p.inv_rows_per_image);
-            int r = m - n * p.rows_per_image;
-            while (r < 0) {
-                --n;
-                r += p.rows_per_image;
-            }
-            while (r >= p.rows_per_image) {
-                ++n;
-                r -= p.rows_per_image;
-            }
-            const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
-            const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
-            const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
-            const long long out_row =
-                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) +
-                p.out_row_off;
-            int8_t *dst2 = (EXTRAS && p.out2) ? p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w +
-                                              X + p.out2_row_off) * p.out2_pitch
-                                  : nullptr;
-            const int8_t *skip = (EXTRAS && p.skip) ? p.skip + ((long long)n * p.out_h * p.out_w + Y * p.out_w + X) *
-                                                       p.skip_pitch
-                                        : nullptr;
-            const int col0 = nt * p.n_tile;
-            int8_t *dst = p.out + out_row * p.out_pitch +
-                          ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
-            float *ldst = p.logits_mode ? p.logits + (long long)m * p.n_actions : nullptr;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) +
-                                   (uint32_t)(a * acc_stride + sub * acc_cols);
-            for (int c0 = c_begin; c0 < c_end; c0 += 16) {
-                int acc[16];
-                {
-                    TRACE_T0();
-                    tmem_ld16(taddr + c0, acc);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(7);
-                }
-                if (c0 + 16 >= c_end && sub == SUB - 1) {
-                    // all of this warp's reads of the stage are done: hand it back to the MMA warp
-                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(acc_empty0 + 8 * a);
-                }
-                if (!valid) continue;
-                if (EXTRAS && skip) {  // residual add in the int32 domain
-                    const uint4 sv = __ldg(reinterpret_cast<const uint4 *>(skip + col0 + c0));
-                    const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        acc[i] += s_skip_mul[col0 + c0 + i] * (int)(int8_t)(sw[i >> 2] >> (8 * (i & 3)));
-                }
-                float ks[16], bs[16];
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const float4 kv = *reinterpret_cast<const float4 *>(&s_ks[col0 + c0 + 4 * g]);
-                    const float4 bv = *reinterpret_cast<const float4 *>(&s_bs[col0 + c0 + 4 * g]);
-                    ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
-                    bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
-                }
-                if (ldst) {
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (col0 + c0 + i < p.n_actions)
-                            ldst[col0 + c0 + i] = epilogue_float(acc[i], ks[i], bs[i], false);
-                } else {
-                    uint32_t w[4];
-                    if (p.fast_div) {
-                        if (p.relu_out) requant16_fastdiv<true>(acc, ks, bs, p.s_out, p.inv_s_out, w);
-                        else requant16_fastdiv<false>(acc, ks, bs, p.s_out, p.inv_s_out, w);
-                    } else {
-                        requant16(acc, ks, bs, p.relu_out != 0, p.s_out, p.inv_s_out, w);
-                    }
-                    if (EXTRAS && (p.out_relu | p.out2_relu)) {
-                        uint32_t wr[4];
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
-                            const uint32_t neg = w[g] & 0x80808080u;
-                            wr[g] = w[g] & ~(neg | (neg - (neg >> 7)));
-                        }
-                        *reinterpret_cast<uint4 *>(dst + c0) =
-                            p.out_relu ? make_uint4(wr[0], wr[1], wr[2], wr[3])
-                                       : make_uint4(w[0], w[1], w[2], w[3]);
-                        if (dst2)
-                            *reinterpret_cast<uint4 *>(dst2 + col0 + c0) =
-                                p.out2_relu ? make_uint4(wr[0], wr[1], wr[2], wr[3])
-                                            : make_uint4(w[0], w[1], w[2], w[3]);
-                    } else {
-                        *reinterpret_cast<uint4 *>(dst + c0) = make_uint4(w[0], w[1], w[2], w[3]);
-                        if (EXTRAS && dst2)
-                            *reinterpret_cast<uint4 *>(dst2 + col0 + c0) = make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                }
-            }
-            }  // sub
+        EpiCtx c;
+        c.tmem_base = tmem_base;
+        c.acc_full0 = acc_full0;
+        c.acc_empty0 = acc_empty0;
+        c.total_tiles = total_tiles;
+        c.n_acc = n_acc;
+        c.acc_stride = acc_stride;
+        c.acc_cols = acc_cols;
+        c.sub = SUB;
+        c.s_ks = s_ks;
+        c.s_bs = s_bs;
+        c.s_skip_mul = s_skip_mul;
+        c.abort_flag = abort_flag;
+        if (p.logits_mode) epilogue_role<false, kEpiLogits, false>(p, c, warp, lane);
+        else if (p.fast_div) {
+            if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true>(p, c, warp, lane);
+            else epilogue_role<EXTRAS, kEpiFastDiv, false>(p, c, warp, lane);
+        } else {
+            if (p.relu_out) epilogue_role<EXTRAS, kEpiTieCheck, true>(p, c, warp, lane);
+            else epilogue_role<EXTRAS, kEpiTieCheck, false>(p, c, warp, lane);
         }
     }
 
