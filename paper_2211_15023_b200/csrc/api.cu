@@ -311,6 +311,10 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             ACCERL_CUDA_TRY(launch_mlp_fused(p, (const float *)obs_dev, uniforms_dev, B, logits_dev,
                                              actions_dev, logp_dev, st));
             break;
+        case Step::FC_SAMPLE:
+            ACCERL_CUDA_TRY(launch_fc_sample(p->fc_sample, uniforms_dev, B, logits_dev, actions_dev, logp_dev,
+                                             p->sm_count, st));
+            break;
         case Step::SAMPLE:
             ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev,
                                           logp_dev, st));

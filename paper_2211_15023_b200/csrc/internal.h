@@ -51,7 +51,7 @@ struct LayerPlan {
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
     enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED,
-                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4 } kind;
+                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4, FC_SAMPLE } kind;
     int layer = -1;
     int tc = -1;  // index into accerl_policy::tc_steps (TC_GEMM) or ::pools (POOL_DUAL)
     std::string kernel, covers;
@@ -67,6 +67,14 @@ struct TcStep {
 };
 
 struct MlpFusedParams;  // mlp_fused.cu
+
+// last FC layer fused with the sampler (fc_sample.cu)
+struct FcSampleParams {
+    const int8_t *x;  // [B][pitch] int8 input rows
+    int pitch, k4, n_actions;
+    const int32_t *w;  // [k4][32] words, lane = action
+    const float *kscale, *bias;
+};
 
 // max-pool that writes a plain NHWC output and / or a padded-border one (tc_mixed_plan.cu)
 struct PoolDualParams {
@@ -107,6 +115,7 @@ struct accerl_policy {
     int in_pad4_w = 0;
     std::vector<accerl::TapDesc> taps;    // per tensor (index t + 1); empty or null ptr = generic buffer
     std::shared_ptr<accerl::MlpFusedParams> mlp;  // set when the whole step is one fused launch
+    accerl::FcSampleParams fc_sample = {};         // used by a Step::FC_SAMPLE launch
     std::vector<int> tensor_s2d;          // space-to-depth factor of tensor t at [t + 1]
     int sm_count = 0;
     std::vector<accerl::DeviceBuf> bufs;  // bufs[0] holds the quantised input
@@ -158,5 +167,10 @@ accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, 
 cudaError_t launch_mlp_fused(const accerl_policy *p, const float *obs, const float *u, int B,
                              float *logits, int32_t *actions, float *logp, cudaStream_t st);
 accerl_status upload_bytes(accerl_policy *p, const void *host, size_t bytes, void **dev);
+bool fc_sample_fits(const accerl_policy *p, const accerl_layer_desc *layers, int n_layers, int i);
+accerl_status build_fc_sample(accerl_policy *p, const accerl_layer_desc &d, int layer, const int8_t *x,
+                              int pitch, Step *out);
+cudaError_t launch_fc_sample(const FcSampleParams &q, const float *u, int B, float *logits,
+                             int32_t *actions, float *logp, int sm_count, cudaStream_t st);
 
 }  // namespace accerl

@@ -271,6 +271,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         return ACCERL_OK;
     };
     std::vector<Step> steps;
+    bool fused_sample = false;
     p->taps.assign(n_layers + 1, TapDesc());
     {
         Step s0;
@@ -327,6 +328,13 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             s.tc = (int)p->pools.size() - 1;
             s.kernel = "maxpool_dual_kernel";
             steps.push_back(s);
+            continue;
+        }
+        if (role[i] == TCFC && fin.plain && fc_sample_fits(p, layers, n_layers, i)) {
+            // the last layer runs fused with the sampler
+            if ((st = build_fc_sample(p, d, i, fin.p_plain, L.in_c, &s)) != ACCERL_OK) return st;
+            steps.push_back(s);
+            fused_sample = true;
             continue;
         }
         // ---- tensor-core layer
@@ -528,11 +536,13 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if (g.fast_div) s.kernel += "[3-step divide verified]";
         steps.push_back(s);
     }
-    Step ss;
-    ss.kind = Step::SAMPLE;
-    ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
-    ss.covers = "sample";
-    steps.push_back(ss);
+    if (!fused_sample) {
+        Step ss;
+        ss.kind = Step::SAMPLE;
+        ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
+        ss.covers = "sample";
+        steps.push_back(ss);
+    }
     p->steps = steps;
     *used = true;
     return ACCERL_OK;

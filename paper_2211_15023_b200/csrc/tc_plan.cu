@@ -258,6 +258,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
     p->tensor_s2d[n_layers] = 1;
 
     std::vector<Step> steps;
+    bool fused_sample = false;
     Step s0;
     s0.kind = Step::INGEST_S2D;
     s0.kernel = (p->in_c == 4 && p->tensor_s2d[0] == 4) ? "ingest_u8_s2d44_kernel"
@@ -268,6 +269,14 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
     for (int i = 0; i < n_layers; ++i) {
         const accerl_layer_desc &d = layers[i];
         const LayerPlan &L = p->layers[i];
+        if (fc_sample_fits(p, layers, n_layers, i)) {  // the last layer runs fused with the sampler
+            Step fs;
+            accerl_status fst = build_fc_sample(p, d, i, p->bufs[L.in_buf].ptr, L.in_c, &fs);
+            if (fst != ACCERL_OK) return fst;
+            steps.push_back(fs);
+            fused_sample = true;
+            continue;
+        }
         TcStep ts;
         memset(&ts.prm, 0, sizeof(ts.prm));
         TcGemmParams &g = ts.prm;
@@ -400,11 +409,13 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         s.covers = "layer " + std::to_string(i);
         steps.push_back(s);
     }
-    Step ss;
-    ss.kind = Step::SAMPLE;
-    ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
-    ss.covers = "sample";
-    steps.push_back(ss);
+    if (!fused_sample) {
+        Step ss;
+        ss.kind = Step::SAMPLE;
+        ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
+        ss.covers = "sample";
+        steps.push_back(ss);
+    }
     p->steps = steps;
     *used = true;
     return ACCERL_OK;
