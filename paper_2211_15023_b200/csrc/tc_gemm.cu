@@ -247,10 +247,13 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 r -= p.rows_per_image;
             }
             const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
-            const bool valid = n < p.batch && Y < p.out_h && X < p.out_w;
+            const int first_px = X * p.px_per_row;  // 0 unless the row holds several pixels
+            const bool valid = n < p.batch && Y < p.out_h && (p.px_per_row ? first_px < p.px_w : X < p.out_w);
+            // columns to store: all, or those of the pixels inside the image
+            const int n_store = p.px_per_row ? min(c_end, (p.px_w - first_px) * p.px_cols) : c_end;
             const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
             const long long out_row =
-                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) +
+                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) * p.out_xmul +
                 p.out_row_off;
             int8_t *dst = p.out + out_row * p.out_pitch +
                           ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
@@ -258,10 +261,11 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
             const int8_t *skip = nullptr;
             if (EXTRAS) {
                 if (has_out2)
-                    dst2 = p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w + X +
-                                     p.out2_row_off) * p.out2_pitch + col0;
+                    dst2 = p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w +
+                                     X * p.out2_xmul + p.out2_row_off) * p.out2_pitch + col0;
                 if (has_skip)
-                    skip = p.skip + ((long long)n * p.out_h * p.out_w + Y * p.out_w + X) * p.skip_pitch + col0;
+                    skip = p.skip + ((long long)n * p.skip_rows_per_image + Y * p.skip_grid_w +
+                                     X * p.skip_xmul + p.skip_row_off) * p.skip_pitch + col0;
             }
             float *ldst = MODE == kEpiLogits ? p.logits + (long long)m * p.n_actions : nullptr;
             const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) +
@@ -282,7 +286,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 }
                 if (EXTRAS && has_skip) {  // residual add in the int32 domain
                     uint4 sv = make_uint4(0, 0, 0, 0);
-                    if (valid) sv = __ldg(reinterpret_cast<const uint4 *>(skip + c0));
+                    if (valid && c0 < n_store) sv = __ldg(reinterpret_cast<const uint4 *>(skip + c0));
                     const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
@@ -320,11 +324,11 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                         }
                         relu = make_uint4(wr[0], wr[1], wr[2], wr[3]);
                     }
-                    if (valid) {
+                    if (valid && c0 < n_store) {
                         *reinterpret_cast<uint4 *>(dst + c0) = p.out_relu ? relu : plain;
                         if (has_out2) *reinterpret_cast<uint4 *>(dst2 + c0) = p.out2_relu ? relu : plain;
                     }
-                } else if (valid) {
+                } else if (valid && c0 < n_store) {
                     *reinterpret_cast<uint4 *>(dst + c0) = plain;
                 }
             }
@@ -360,7 +364,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int CH = p.chunk_bytes;
     const int a_chunk_bytes = kTileM * CH;
-    const int b_tile_bytes = p.n_tile * CH;
+    const int CHB = p.kstep_list ? 32 : CH;  // bytes of a weight row per chunk
+    const int b_tile_bytes = p.n_tile * CHB;
     // shifted mode: a stage is one box of a_rows rows that all taps of the tile read at row offsets
     // sub > 1 (shifted mode only): a pipeline step covers `sub` consecutive 128-row tiles, one TMA
     // box and one accumulator each, so that the barrier round trips are paid once per step
@@ -376,11 +381,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     volatile int *abort_flag = &bars.abort_flag;
 
     {
-        const int ks_per_chunk = CH / 32;
+        const int ks_per_chunk = p.kstep_list ? 1 : CH / 32;
         const int Gt = p.shifted ? p.n_chunks : p.group;
         for (int t = threadIdx.x; t < p.n_chunks * ks_per_chunk; t += blockDim.x) {
             const int j = t / ks_per_chunk, k = t - j * ks_per_chunk, cl = j % Gt;
-            const uint32_t a_rel = (uint32_t)(p.shifted ? p.row_off[j] * CH : cl * a_chunk_bytes);
+            const uint32_t a_rel = (uint32_t)(p.shifted ? p.row_off[j] * CH + (p.kstep_list ? p.col_off[j] : 0)
+                                                        : cl * a_chunk_bytes);
             const uint32_t b_rel =
                 RESIDENT_B ? smem_u32(resident_b) + (uint32_t)(j * b_tile_bytes)
                            : (uint32_t)(Gt * a_chunk_bytes + cl * b_tile_bytes);
@@ -510,8 +516,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint64_t desc_hi =
             (uint64_t)(((uint32_t)(8 * CH) >> 4) | (1u << 14) |
                        ((CH == 128 ? 2u : (CH == 64 ? 4u : 6u)) << 29)) << 32;
+        const uint64_t desc_hi_b =
+            (uint64_t)(((uint32_t)(8 * CHB) >> 4) | (1u << 14) |
+                       ((CHB == 128 ? 2u : (CHB == 64 ? 4u : 6u)) << 29)) << 32;
         const uint32_t desc_lo_flags = 1u << 16;
-        const int k_steps = CH / 32;
+        const int k_steps = p.kstep_list ? 1 : CH / 32;
         bool ok = true;
         if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
         int a = mw, base_slot = 0;
@@ -550,7 +559,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         for (int t = t0; t < t1; ++t) {
                             const uint2 rel = s_desc[t];
                             const uint32_t b_lo = RESIDENT_B ? rel.y : st_lo + rel.y;
-                            mma_i8(d_tmem + sub * acc_cols, desc_hi | (sub_lo + rel.x), desc_hi | b_lo,
+                            mma_i8(d_tmem + sub * acc_cols, desc_hi | (sub_lo + rel.x), desc_hi_b | b_lo,
                                    idesc, (uint32_t)t);
                         }
                     }
@@ -667,7 +676,7 @@ accerl_status tc_make_map(void *map_out, const void *base, long long rows, int r
 
 size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
 {
-    const int a_chunk = kTileM * p.chunk_bytes, b_tile = p.n_tile * p.chunk_bytes;
+    const int a_chunk = kTileM * p.chunk_bytes, b_tile = p.n_tile * (p.kstep_list ? 32 : p.chunk_bytes);
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
     const size_t stage = p.shifted ? p.sub * (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
                                    : (size_t)p.group * (a_chunk + (resident_b ? 0 : b_tile));
@@ -698,6 +707,9 @@ bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
         p.n_acc_stages = pow2_floor(std::min(kTcMaxAccStages, 512 / (sub * acc_cols)));
         if (p.n_acc_stages < 1) continue;
         p.n_mma = std::min(kMmaWarps, p.n_acc_stages);
+        // wide accumulators leave only two to four stages: give every issuing warp two of them, so
+        // that it works on the next tile while the epilogue drains the previous one
+        if (sub == 1 && p.shifted && acc_cols >= 128 && p.n_acc_stages >= 2) p.n_mma = p.n_acc_stages / 2;
         const int want = sub > 1 ? 2 * p.n_mma : std::max(2, p.n_mma);
         if (sub > 1 && p.n_acc_stages < 2 * p.n_mma) continue;
         for (int s = kTcMaxStages / p.n_mma * p.n_mma; s >= want; s -= p.n_mma) {

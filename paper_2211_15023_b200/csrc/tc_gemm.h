@@ -17,6 +17,9 @@ struct TcGemmParams {
     // [j * n_total, (j + 1) * n_total) of the packed weight tensor
     int n_chunks, chunk_bytes;
     int row_off[kTcMaxChunks], col_off[kTcMaxChunks];
+    // kstep_list = 1 (shifted mode only): "chunk" j is ONE 32-byte K step, read at byte col_off[j]
+    // of row row0 + row_off[j] of the A box; the weights are packed [j][n_total][32 bytes]
+    int kstep_list;
     // tiling
     int m_tiles, n_tiles, n_tile, n_total;
     int n_stages, n_acc_stages, n_acc_log2, tmem_cols;
@@ -33,15 +36,21 @@ struct TcGemmParams {
     int out_s2d, out_rows_per_image, out_grid_w, out_pitch;
     int out_s2d_log2;
     int out_row_off;  // added to the output row (a one-pixel border of a padded consumer layout)
+    // Several pixels per GEMM row (px_per_row > 0): row (Y, X) holds output pixels
+    // X * px_per_row + j, j < px_per_row, px_cols columns each; pixels at or beyond px_w are not
+    // stored.  out_xmul scales X in the output row (px_per_row when out_pitch is one pixel).
+    int px_per_row, px_cols, px_w;
+    int out_xmul, out2_xmul;
     int out_relu;     // clamp the stored codes at 0 (the only reader applies ReLU to its input)
     // optional second copy of the output in another layout: row = n * out2_rows_per_image +
     // Y * out2_grid_w + X + out2_row_off, `out2_pitch` bytes apart, ReLU'd if out2_relu
     int8_t *out2;
     int out2_rows_per_image, out2_grid_w, out2_row_off, out2_pitch, out2_relu;
-    // optional residual: acc += skip_mul[c] * skip[n, Y, X, c] from a plain NHWC tensor
+    // optional residual: acc += skip_mul[c] * skip[row][c], row = n * skip_rows_per_image +
+    // Y * skip_grid_w + X * skip_xmul + skip_row_off, rows skip_pitch bytes apart
     const int8_t *skip;
     const int32_t *skip_mul;
-    int skip_pitch;
+    int skip_pitch, skip_rows_per_image, skip_grid_w, skip_xmul, skip_row_off;
     float inv_rows_per_image;  // 1 / rows_per_image, for the division-free row decode
     unsigned grid_w_magic;     // ceil(2^32 / grid_w)
     // epilogue

@@ -345,6 +345,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         const int n_total = role[i] == TCFIRST ? 8 * d.out_c : round_up(d.out_c, 16);
         g.sub = 1;
         g.max_sub = 1;
+        g.out_xmul = g.out2_xmul = 1;
         g.n_total = n_total;
         g.n_tile = n_total > 256 ? 256 : n_total;
         g.n_tiles = n_total / g.n_tile;
@@ -489,6 +490,10 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             g.skip = forms[d.skip_from + 1].p_plain;
             g.skip_mul = L.skip_mul;
             g.skip_pitch = p->layers[d.skip_from].out_cp;
+            g.skip_rows_per_image = L.out_h * L.out_w;
+            g.skip_grid_w = L.out_w;
+            g.skip_xmul = 1;
+            g.skip_row_off = 0;
         }
         g.kscale = ks_dev;
         g.bias = bs_dev;

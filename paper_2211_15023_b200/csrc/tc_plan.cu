@@ -282,6 +282,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         TcGemmParams &g = ts.prm;
         g.sub = 1;
         g.max_sub = 1;
+        g.out_xmul = g.out2_xmul = 1;
         const bool logits = (d.flags & ACCERL_LOGITS) != 0;
         const int n_total = round_up(d.out_c, 16);
         g.n_total = n_total;
