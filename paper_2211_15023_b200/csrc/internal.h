@@ -77,11 +77,18 @@ struct FcSampleParams {
 };
 
 // max-pool that writes a plain NHWC output and / or a padded-border one (tc_mixed_plan.cu)
+struct PoolOut {  // one stored form of the pooled tensor
+    int8_t *ptr;                 // null: unused
+    int hpitch, wpitch;          // stored rows per image, pixels per stored row
+    int off_y, off_x;            // where pixel (0, 0) sits
+    int pix_bytes;               // bytes between stored pixels (>= C)
+    int relu;                    // store max(code, 0)
+};
 struct PoolDualParams {
-    const int8_t *in;
-    int8_t *out_plain, *out_pad;
-    int H, W, C, OH, OW, k, stride, pad_pitch, pad_relu;
-    int in_wpitch;  // pixels per stored input row (>= W)
+    const int8_t *in;            // pixels of C bytes
+    int in_hpitch, in_wpitch, in_off_y, in_off_x;
+    int H, W, C, OH, OW, k, stride;
+    PoolOut out[2];
 };
 
 // where the parity tap of a tensor lives when it is not in the generic plan's buffer

@@ -193,17 +193,41 @@ struct EpiCtx {
     const float *s_ks, *s_bs;
     const int *s_skip_mul;
     volatile int *abort_flag;
+    uint8_t *staging;  // kStagingBytes per epilogue warp when the layer stores through shared memory
 };
 
 enum { kEpiFastDiv = 0, kEpiTieCheck = 1, kEpiLogits = 2 };
+constexpr int kStagingBytes = 32 * 128;  // 32 rows of 128 output bytes
+
+// byte offset of 16-byte piece `ch` of row `row` in a warp's staging tile; the XOR spreads a
+// warp's pieces over the banks both when lanes are rows and when eight lanes share a row
+__device__ __forceinline__ int stage_off(int row, int ch) { return row * 128 + ((ch ^ (row & 7)) << 4); }
+
+__device__ __forceinline__ uint4 relu_codes(uint4 v)
+{
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
+        const uint32_t neg = w[g] & 0x80808080u;
+        w[g] &= ~(neg | (neg - (neg >> 7)));
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
 
 // Epilogue role (warps 8..23): drain accumulators, requantise, store.  The per-layer switches are
 // template parameters, chosen once per launch, so that the loop over 16-column pieces is straight
 // line code: the epilogue is bound by instruction issue.  Rows that are no output position are
 // computed like the others and only their stores are skipped, which keeps the warp converged.
-template <bool EXTRAS, int MODE, bool RELU>
+//
+// STAGED (tiles of 128 columns whose rows are 128 contiguous output bytes): a lane's 16-byte
+// pieces would each touch a different 128-byte line of global memory, 32 lines per store
+// instruction, and the load/store path then bounds the layer.  Instead every warp collects its 32
+// rows in a shared-memory tile and copies it out with eight lanes per row, full lines per
+// instruction; the residual source comes in the same way.
+template <bool EXTRAS, int MODE, bool RELU, bool PX, bool STAGED>
 __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
 {
+    uint8_t *stage = STAGED ? c.staging + (warp - kProdWarps - kMmaWarps) * kStagingBytes : nullptr;
     const int q = warp & 3;         // this warp's quarter of tensor memory
     const int wg = (warp - kProdWarps - kMmaWarps) >> 2;  // epilogue warpgroup
     const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
@@ -247,14 +271,15 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 r -= p.rows_per_image;
             }
             const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
-            const int first_px = X * p.px_per_row;  // 0 unless the row holds several pixels
-            const bool valid = n < p.batch && Y < p.out_h && (p.px_per_row ? first_px < p.px_w : X < p.out_w);
+            // PX: the row holds px_per_row output pixels of px_cols columns each
+            const int first_px = PX ? X * p.px_per_row : 0;
+            const bool valid = n < p.batch && Y < p.out_h && (PX ? first_px < p.px_w : X < p.out_w);
             // columns to store: all, or those of the pixels inside the image
-            const int n_store = p.px_per_row ? min(c_end, (p.px_w - first_px) * p.px_cols) : c_end;
+            const int n_store = PX ? min(c_end, (p.px_w - first_px) * p.px_cols) : c_end;
             const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
             const long long out_row =
-                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w + (X >> sh) * p.out_xmul +
-                p.out_row_off;
+                (long long)n * p.out_rows_per_image + (Y >> sh) * p.out_grid_w +
+                (PX ? X * p.out_xmul : (X >> sh)) + p.out_row_off;
             int8_t *dst = p.out + out_row * p.out_pitch +
                           ((((Y & smask) << sh) + (X & smask)) * p.n_total) + col0;
             int8_t *dst2 = nullptr;
@@ -262,14 +287,35 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
             if (EXTRAS) {
                 if (has_out2)
                     dst2 = p.out2 + ((long long)n * p.out2_rows_per_image + Y * p.out2_grid_w +
-                                     X * p.out2_xmul + p.out2_row_off) * p.out2_pitch + col0;
+                                     (PX ? X * p.out2_xmul : X) + p.out2_row_off) * p.out2_pitch + col0;
                 if (has_skip)
                     skip = p.skip + ((long long)n * p.skip_rows_per_image + Y * p.skip_grid_w +
-                                     X * p.skip_xmul + p.skip_row_off) * p.skip_pitch + col0;
+                                     (PX ? X * p.skip_xmul : X) + p.skip_row_off) * p.skip_pitch + col0;
             }
             float *ldst = MODE == kEpiLogits ? p.logits + (long long)m * p.n_actions : nullptr;
             const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) +
                                    (uint32_t)(a * c.acc_stride + sub * c.acc_cols);
+            // staged mode: what the lanes that copy this row in and out need to know about it
+            // (offsets in 16-byte units from the tensors' bases; 0 pieces for rows that are no output)
+            const int my_pieces = valid ? n_store >> 4 : 0;
+            uint32_t my_out16 = 0, my_out2_16 = 0, my_skip16 = 0;
+            if (STAGED) {
+                my_out16 = (uint32_t)((dst - p.out) >> 4);
+                if (has_out2) my_out2_16 = (uint32_t)((dst2 - p.out2) >> 4);
+                if (has_skip) {
+                    my_skip16 = (uint32_t)((skip - p.skip) >> 4);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = 4 * i + (lane >> 3), ch = lane & 7;
+                        const uint32_t so = __shfl_sync(0xffffffffu, my_skip16, r);
+                        const int np = __shfl_sync(0xffffffffu, my_pieces, r);
+                        uint4 v = make_uint4(0, 0, 0, 0);
+                        if (ch < np) v = __ldg(reinterpret_cast<const uint4 *>(p.skip) + so + ch);
+                        *reinterpret_cast<uint4 *>(stage + stage_off(r, ch)) = v;
+                    }
+                    __syncwarp();
+                }
+            }
             for (int c0 = c_begin; c0 < c_end; c0 += 16) {
                 int acc[16];
                 {
@@ -286,7 +332,8 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 }
                 if (EXTRAS && has_skip) {  // residual add in the int32 domain
                     uint4 sv = make_uint4(0, 0, 0, 0);
-                    if (valid && c0 < n_store) sv = __ldg(reinterpret_cast<const uint4 *>(skip + c0));
+                    if (STAGED) sv = *reinterpret_cast<const uint4 *>(stage + stage_off(lane, c0 >> 4));
+                    else if (valid && c0 < n_store) sv = __ldg(reinterpret_cast<const uint4 *>(skip + c0));
                     const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
@@ -313,7 +360,9 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 if (MODE == kEpiFastDiv) requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
                 else requant16(acc, ks, bs, RELU, s_out, inv_s_out, w);
                 const uint4 plain = make_uint4(w[0], w[1], w[2], w[3]);
-                if (EXTRAS) {
+                if (STAGED) {
+                    *reinterpret_cast<uint4 *>(stage + stage_off(lane, c0 >> 4)) = plain;
+                } else if (EXTRAS) {
                     uint4 relu = plain;
                     if (p.out_relu | p.out2_relu) {
                         uint32_t wr[4];
@@ -332,6 +381,23 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                     *reinterpret_cast<uint4 *>(dst + c0) = plain;
                 }
             }
+            if (STAGED && MODE != kEpiLogits) {
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = 4 * i + (lane >> 3), ch = lane & 7;
+                    const uint32_t o = __shfl_sync(0xffffffffu, my_out16, r);
+                    const uint32_t o2 = has_out2 ? __shfl_sync(0xffffffffu, my_out2_16, r) : 0u;
+                    const int np = __shfl_sync(0xffffffffu, my_pieces, r);
+                    const uint4 v = *reinterpret_cast<const uint4 *>(stage + stage_off(r, ch));
+                    if (ch < np) {
+                        const uint4 vr = (EXTRAS && (p.out_relu | p.out2_relu)) ? relu_codes(v) : v;
+                        reinterpret_cast<uint4 *>(p.out)[o + ch] = (EXTRAS && p.out_relu) ? vr : v;
+                        if (has_out2) reinterpret_cast<uint4 *>(p.out2)[o2 + ch] = p.out2_relu ? vr : v;
+                    }
+                }
+                __syncwarp();  // the tile is rewritten in the next round
+            }
         }
     }
 }
@@ -340,7 +406,9 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
 
 // EXTRAS compiles in the residual add, the second output and the stored-code ReLU; layers that
 // use none of them run the leaner instantiation (the epilogue is bound by instruction issue).
-template <bool RESIDENT_B, bool EXTRAS>
+// PXK is the kernel for rows of several output pixels; it is kept apart so that its epilogue
+// variants do not weigh on the register allocation of the others.
+template <bool RESIDENT_B, bool EXTRAS, bool PXK>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcGemmParams p)
@@ -595,13 +663,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         c.s_bs = s_bs;
         c.s_skip_mul = s_skip_mul;
         c.abort_flag = abort_flag;
-        if (p.logits_mode) epilogue_role<false, kEpiLogits, false>(p, c, warp, lane);
-        else if (p.fast_div) {
-            if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true>(p, c, warp, lane);
-            else epilogue_role<EXTRAS, kEpiFastDiv, false>(p, c, warp, lane);
+        c.staging = stages + (size_t)n_stages * stage_bytes;
+        if constexpr (PXK) {  // multi-pixel rows: only built for the verified division
+            if (p.staged) {
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, true>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, true>(p, c, warp, lane);
+            } else {
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, false>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, false>(p, c, warp, lane);
+            }
         } else {
-            if (p.relu_out) epilogue_role<EXTRAS, kEpiTieCheck, true>(p, c, warp, lane);
-            else epilogue_role<EXTRAS, kEpiTieCheck, false>(p, c, warp, lane);
+            if (p.logits_mode) epilogue_role<false, kEpiLogits, false, false, false>(p, c, warp, lane);
+            else if (p.fast_div) {
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, false, false>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiFastDiv, false, false, false>(p, c, warp, lane);
+            } else {
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiTieCheck, true, false, false>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiTieCheck, false, false, false>(p, c, warp, lane);
+            }
         }
     }
 
@@ -680,7 +759,7 @@ size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
     const size_t stage = p.shifted ? p.sub * (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
                                    : (size_t)p.group * (a_chunk + (resident_b ? 0 : b_tile));
-    return 1024 + res + (size_t)p.n_stages * stage;
+    return 1024 + res + (size_t)p.n_stages * stage + (p.staged ? (size_t)4 * kEpiGroups * kStagingBytes : 0);
 }
 
 static int pow2_floor(int v)
@@ -740,8 +819,14 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
         kernel<<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, p);
         return cudaSuccess;
     };
-    cudaError_t e = resident_b ? (extras ? go(tc_gemm_kernel<true, true>) : go(tc_gemm_kernel<true, false>))
-                               : (extras ? go(tc_gemm_kernel<false, true>) : go(tc_gemm_kernel<false, false>));
+    cudaError_t e;
+    if (p.px_per_row) {
+        if (!resident_b || !p.fast_div || p.logits_mode) return cudaErrorInvalidValue;
+        e = extras ? go(tc_gemm_kernel<true, true, true>) : go(tc_gemm_kernel<true, false, true>);
+    } else {
+        e = resident_b ? (extras ? go(tc_gemm_kernel<true, true, false>) : go(tc_gemm_kernel<true, false, false>))
+                       : (extras ? go(tc_gemm_kernel<false, true, false>) : go(tc_gemm_kernel<false, false, false>));
+    }
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

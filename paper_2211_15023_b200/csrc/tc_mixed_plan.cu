@@ -1,14 +1,23 @@
 // Tensor-core plan for residual conv stacks (the IMPALA-ResNet shape): 3x3 stride-1 pad-1
-// convolutions with 16 or 32 input channels run on tc_gemm_kernel in shifted mode, the remaining
-// layers (a first conv on 4 channels, max-pools) on CUDA-core kernels.
+// convolutions with 16 or 32 channels run on tc_gemm_kernel in shifted mode, a first conv on
+// 4-channel frames too, max-pools on a CUDA-core kernel.
 //
-// A tensor read by such a conv is stored with a one-pixel zero border and 32 bytes per pixel
-// ([n][H+2][W+2][32], channels 16..31 zero when the tensor has 16), so that the conv is a valid
-// 3x3 conv on the padded image: one GEMM row per padded position, taps at row offsets
-// ky * (W+2) + kx, 32-byte rows = one K step per tap.  Borders and padding channels are zeroed
-// once at create and never written.  A tensor may be kept in two forms at once (for instance the
-// input x of a residual block: plain for the skip add, padded and ReLU'd for the block's first
-// conv); producers (the conv epilogue, the pooling kernel) write both.
+// Wide images (W >= 16), "slot" layout: a tensor is stored [n][H+2][PW][C] with the image at row 1,
+// pixel 1, zero elsewhere, PW a multiple of 8 >= W + 2.  One GEMM row is P consecutive stored
+// pixels (P * C_in = 64 or 128 bytes) and produces the P output pixels above them, N = P * C_out
+// = 128 columns, with banded weights: output pixel j of the row meets stored pixels j .. j + 2 of
+// the rows of the three taps ky, i.e. the P pixels of the GEMM row ky * PW/P further down plus the
+// first two of the row after it.  The K loop is the list of the 32-byte steps that cover those
+// (P + 2) * C_in bytes; most of the weight matrix is zero, but with 16 or 32 output channels the
+// tensor pipe is paid per instruction, not per flop, and a tile of 128 x 128 outputs amortises
+// the epilogue's per-tile work eight times better than 128 x 16.
+//
+// Narrow images, "pad" layout: [n][H+2][W+2][32 bytes] (channels 16..31 zero when the tensor has
+// 16), one GEMM row per padded position, taps at row offsets ky * (W+2) + kx, one K step per tap.
+//
+// Borders and padding are zeroed once at create and never written.  A tensor may be kept in two
+// forms at once (for instance the input x of a residual block: as it is for the skip add, and
+// ReLU'd for the block's first conv); producers (the conv epilogue, the pooling kernel) write both.
 #include <string.h>
 
 #include <algorithm>
@@ -18,7 +27,7 @@
 namespace accerl {
 
 // ---------------------------------------------------------------------------------------
-// max-pool with up to two outputs: plain NHWC and / or padded-border (optionally ReLU'd)
+// max-pool with up to two stored forms of its output (any pitches and offsets, optionally ReLU'd)
 // ---------------------------------------------------------------------------------------
 __global__ void maxpool_dual_kernel(const PoolDualParams q, long long total)
 {
@@ -32,26 +41,38 @@ __global__ void maxpool_dual_kernel(const PoolDualParams q, long long total)
     int oy = (int)(t % q.OH);
     long long n = t / q.OH;
     uint32_t m[4] = {0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u};
-    for (int ky = 0; ky < q.k; ++ky)
-        for (int kx = 0; kx < q.k; ++kx) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(
-                q.in + ((n * q.H + oy * q.stride + ky) * q.in_wpitch + ox * q.stride + kx) * q.C + g * 16));
-            m[0] = __vmaxs4(m[0], v.x);
-            m[1] = __vmaxs4(m[1], v.y);
-            m[2] = __vmaxs4(m[2], v.z);
-            m[3] = __vmaxs4(m[3], v.w);
-        }
-    if (q.out_plain)
-        *reinterpret_cast<uint4 *>(q.out_plain + ((n * q.OH + oy) * q.OW + ox) * q.C + g * 16) =
-            make_uint4(m[0], m[1], m[2], m[3]);
-    if (q.out_pad) {
-        if (q.pad_relu) {
+    const int8_t *win = q.in + ((n * q.in_hpitch + oy * q.stride + q.in_off_y) * q.in_wpitch + ox * q.stride +
+                                q.in_off_x) * q.C + g * 16;
+    const int row_bytes = q.in_wpitch * q.C;
+    if (q.k == 3) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) m[i] = __vmaxs4(m[i], 0u);
-        }
-        const long long row = (n * (q.OH + 2) + oy + 1) * (q.OW + 2) + ox + 1;
-        *reinterpret_cast<uint4 *>(q.out_pad + row * q.pad_pitch + g * 16) =
-            make_uint4(m[0], m[1], m[2], m[3]);
+        for (int ky = 0; ky < 3; ++ky)
+#pragma unroll
+            for (int kx = 0; kx < 3; ++kx) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(win + ky * row_bytes + kx * q.C));
+                m[0] = __vmaxs4(m[0], v.x);
+                m[1] = __vmaxs4(m[1], v.y);
+                m[2] = __vmaxs4(m[2], v.z);
+                m[3] = __vmaxs4(m[3], v.w);
+            }
+    } else {
+        for (int ky = 0; ky < q.k; ++ky)
+            for (int kx = 0; kx < q.k; ++kx) {
+                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(win + ky * row_bytes + kx * q.C));
+                m[0] = __vmaxs4(m[0], v.x);
+                m[1] = __vmaxs4(m[1], v.y);
+                m[2] = __vmaxs4(m[2], v.z);
+                m[3] = __vmaxs4(m[3], v.w);
+            }
+    }
+#pragma unroll
+    for (int o = 0; o < 2; ++o) {
+        const PoolOut &po = q.out[o];
+        if (!po.ptr) continue;
+        uint4 v = make_uint4(m[0], m[1], m[2], m[3]);
+        if (po.relu) v = make_uint4(__vmaxs4(m[0], 0u), __vmaxs4(m[1], 0u), __vmaxs4(m[2], 0u), __vmaxs4(m[3], 0u));
+        *reinterpret_cast<uint4 *>(po.ptr + ((n * po.hpitch + oy + po.off_y) * po.wpitch + ox + po.off_x) * po.pix_bytes +
+                                   g * 16) = v;
     }
 }
 
@@ -130,13 +151,31 @@ cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t
 // ---------------------------------------------------------------------------------------
 namespace {
 
-enum Role { GENERIC, POOL, TCCONV, TCFC, TCFIRST };
+enum Role { GENERIC, POOL, TCCONV, TCPX, TCFC, TCFIRST };
 
 struct Forms {  // which stored forms of a tensor its readers need
-    bool plain = false, plain_relu = false, pad = false, pad_relu = false;
-    int8_t *p_plain = nullptr, *p_plain_relu = nullptr, *p_pad = nullptr;
-    int count() const { return (plain ? 1 : 0) + (plain_relu ? 1 : 0) + ((pad || pad_relu) ? 1 : 0); }
+    bool plain = false, plain_relu = false, pad = false, pad_relu = false, slot = false, slot_relu = false;
+    int8_t *p_plain = nullptr, *p_plain_relu = nullptr, *p_pad = nullptr, *p_slot = nullptr,
+           *p_slot_relu = nullptr;
+    int count() const
+    {
+        return (plain ? 1 : 0) + (plain_relu ? 1 : 0) + ((pad || pad_relu) ? 1 : 0) + (slot ? 1 : 0) +
+               (slot_relu ? 1 : 0);
+    }
 };
+
+int slot_pw(int W) { return round_up(W + 2, 8); }
+
+// pixels per GEMM row of a multi-pixel conv, 0 if the layer does not qualify
+int tcpx_pixels(const accerl_layer_desc &d)
+{
+    if (d.kind != ACCERL_CONV2D || d.kh != 3 || d.kw != 3 || d.stride != 1 || d.pad != 1) return 0;
+    if ((d.in_c != 16 && d.in_c != 32) || (d.out_c != 16 && d.out_c != 32) || d.in_w < 16) return 0;
+    const int P = 128 / d.out_c, row = P * d.in_c;
+    if (row != 64 && row != 128) return 0;
+    if (128 + 2 * (slot_pw(d.in_w) / P) + 1 > 248) return 0;
+    return P;
+}
 
 bool tcconv_ok(const accerl_layer_desc &d)
 {
@@ -171,7 +210,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         const accerl_layer_desc &d = layers[i];
         const LayerPlan &L = p->layers[i];
         if (tcconv_ok(d)) {
-            role[i] = TCCONV;
+            role[i] = tcpx_pixels(d) ? TCPX : TCCONV;
             ++n_tc;
         } else if (d.kind == ACCERL_MAXPOOL && (d.in_c == 16 || d.in_c == 32) && d.pad == 0) {
             role[i] = POOL;
@@ -194,12 +233,17 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         } else {
             return ACCERL_OK;
         }
-        if (d.skip_from >= 0 && role[i] != TCCONV) return ACCERL_OK;
+        if (d.skip_from >= 0 && role[i] != TCCONV && role[i] != TCPX) return ACCERL_OK;
     }
     if (n_tc == 0) return ACCERL_OK;
     for (int i = 0; i < n_layers; ++i)
         if ((long long)p->max_batch * (p->layers[i].in_h + 2) * (p->layers[i].in_w + 2) + 512 >= (1LL << 31))
             return ACCERL_OK;
+
+    // A multi-pixel conv cannot write the pad layout of a 16-channel tensor (its pixels are not
+    // contiguous there): such a layer falls back to one position per GEMM row.
+    for (int i = 0; i + 1 < n_layers; ++i)
+        if (role[i] == TCPX && role[i + 1] == TCCONV) role[i] = TCCONV;
 
     // ---- forms of every tensor (index t + 1; tensor -1 is the quantised input)
     std::vector<Forms> forms(n_layers + 1);
@@ -211,24 +255,35 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         const accerl_layer_desc &d = layers[j];
         Forms &f = forms[j];  // tensor j - 1
         const bool relu_in = (d.flags & ACCERL_RELU_IN) && !(layers[j - 1].flags & ACCERL_RELU_OUT);
-        if (role[j] == GENERIC || role[j] == POOL) {
+        if (role[j] == GENERIC) {
             if (relu_in) return ACCERL_OK;
             f.plain = true;
+        } else if (role[j] == POOL) {
+            if (relu_in) return ACCERL_OK;
+            // a pool reads whatever its producer writes naturally
+            (role[j - 1] == TCPX ? f.slot : f.plain) = true;
         } else if (role[j] == TCCONV) {
             (relu_in ? f.pad_relu : f.pad) = true;
+        } else if (role[j] == TCPX) {
+            (relu_in ? f.slot_relu : f.slot) = true;
         } else {
             (relu_in ? f.plain_relu : f.plain) = true;
         }
-        if (d.skip_from >= 0) forms[d.skip_from + 1].plain = true;
+        if (d.skip_from >= 0) {
+            Forms &fs = forms[d.skip_from + 1];
+            (role[j] == TCPX ? fs.slot : fs.plain) = true;
+        }
     }
     for (int t = 0; t < n_layers; ++t) {
         Forms &f = forms[t];
         if (f.pad && f.pad_relu) return ACCERL_OK;
-        if (keep && !f.plain && !f.pad) f.plain = true;  // the parity tap needs an un-ReLU'd form
+        if (keep && !f.plain && !f.pad && !f.slot) f.plain = true;  // the parity tap needs an un-ReLU'd form
         if (f.count() > 2) return ACCERL_OK;
         if (t > 0 && (role[t - 1] == GENERIC || role[t - 1] == TCFIRST) && (f.count() != 1 || !f.plain))
             return ACCERL_OK;
         if (t > 0 && role[t - 1] == POOL && f.plain_relu) return ACCERL_OK;
+        if (t > 0 && role[t - 1] == TCPX && (f.pad || f.pad_relu) && layers[t - 1].out_c != 32)
+            return ACCERL_OK;
     }
 
     // ---- buffers: plain forms live in the generic plan's buffers, the others are new
@@ -246,6 +301,9 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if ((f.pad || f.pad_relu) &&
             (st = alloc_zeroed(p, (size_t)p->max_batch * (H + 2) * (W + 2) * 32, &f.p_pad)) != ACCERL_OK)
             return st;
+        const size_t slot_bytes = (size_t)p->max_batch * (H + 2) * slot_pw(W) * C;
+        if (f.slot && (st = alloc_zeroed(p, slot_bytes, &f.p_slot)) != ACCERL_OK) return st;
+        if (f.slot_relu && (st = alloc_zeroed(p, slot_bytes, &f.p_slot_relu)) != ACCERL_OK) return st;
     }
 
     // ---- first conv on tensor cores: frames stored as [n][H+2][PW][4 B] with the image at row 1,
@@ -297,13 +355,20 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         Step s;
         s.layer = i;
         s.covers = "layer " + std::to_string(i);
-        if (i + 1 < n_layers && !fout.plain && (fout.pad || fout.pad_relu) && !fout.pad_relu) {
+        if (i + 1 < n_layers && !fout.plain && fout.pad) {
             // parity tap from the padded, un-ReLU'd form
             TapDesc &td = p->taps[i + 1];
             td.ptr = fout.p_pad;
             td.pitch = 32;
             td.hpitch = L.out_h + 2;
             td.wpitch = L.out_w + 2;
+            td.off_y = td.off_x = 1;
+        } else if (i + 1 < n_layers && !fout.plain && fout.slot) {
+            TapDesc &td = p->taps[i + 1];
+            td.ptr = fout.p_slot;
+            td.pitch = L.out_cp;
+            td.hpitch = L.out_h + 2;
+            td.wpitch = slot_pw(L.out_w);
             td.off_y = td.off_x = 1;
         }
         if (role[i] == GENERIC) {
@@ -315,12 +380,30 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if (role[i] == POOL) {
             PoolDualParams q;
             memset(&q, 0, sizeof(q));
-            q.in = (i == 1 && role[0] == TCFIRST) ? first_out : fin.p_plain;
-            q.in_wpitch = (i == 1 && role[0] == TCFIRST) ? OW8 * 8 : L.in_w;
-            q.out_plain = fout.plain ? fout.p_plain : nullptr;
-            q.out_pad = fout.p_pad;
-            q.pad_relu = fout.pad_relu ? 1 : 0;
-            q.pad_pitch = 32;
+            if (i == 1 && role[0] == TCFIRST) {
+                q.in = first_out;
+                q.in_hpitch = L.in_h;
+                q.in_wpitch = OW8 * 8;
+            } else if (fin.slot) {
+                q.in = fin.p_slot;
+                q.in_hpitch = L.in_h + 2;
+                q.in_wpitch = slot_pw(L.in_w);
+                q.in_off_y = q.in_off_x = 1;
+            } else {
+                q.in = fin.p_plain;
+                q.in_hpitch = L.in_h;
+                q.in_wpitch = L.in_w;
+            }
+            int n_po = 0;
+            const int OH = L.out_h, OW = L.out_w, C = L.in_c;
+            if (fout.plain) q.out[n_po++] = PoolOut{fout.p_plain, OH, OW, 0, 0, C, 0};
+            if (fout.pad || fout.pad_relu)
+                q.out[n_po++] = PoolOut{fout.p_pad, OH + 2, OW + 2, 1, 1, 32, fout.pad_relu ? 1 : 0};
+            if (fout.slot && n_po < 2) q.out[n_po++] = PoolOut{fout.p_slot, OH + 2, slot_pw(OW), 1, 1, C, 0};
+            else if (fout.slot) return bail();
+            if (fout.slot_relu && n_po < 2)
+                q.out[n_po++] = PoolOut{fout.p_slot_relu, OH + 2, slot_pw(OW), 1, 1, C, 1};
+            else if (fout.slot_relu) return bail();
             q.H = L.in_h; q.W = L.in_w; q.C = L.in_c; q.OH = L.out_h; q.OW = L.out_w;
             q.k = d.kh; q.stride = d.stride;
             p->pools.push_back(q);
@@ -342,7 +425,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         memset(&ts.prm, 0, sizeof(ts.prm));
         TcGemmParams &g = ts.prm;
         const bool logits = (d.flags & ACCERL_LOGITS) != 0;
-        const int n_total = role[i] == TCFIRST ? 8 * d.out_c : round_up(d.out_c, 16);
+        const int P = role[i] == TCPX ? tcpx_pixels(d) : 0;  // output pixels per GEMM row
+        const int n_total = role[i] == TCFIRST ? 8 * d.out_c : (P ? P * d.out_c : round_up(d.out_c, 16));
         g.sub = 1;
         g.max_sub = 1;
         g.out_xmul = g.out2_xmul = 1;
@@ -354,6 +438,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         long long a_rows_total;
         int row_bytes;
         const float *ks_dev = L.kscale, *bs_dev = L.bias;
+        const int32_t *px_skip_mul = nullptr;
         if (role[i] == TCFIRST) {
             // GEMM row = 8 consecutive padded pixels (32 B); output column j * out_c + oc is output
             // pixel j of the group.  Input pixel (row ky, offset d8 * 8 + pin from the group's
@@ -396,6 +481,58 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             if ((st = upload_bytes(p, bs.data(), bs.size() * 4, &bd)) != ACCERL_OK) return st;
             ks_dev = (const float *)kd;
             bs_dev = (const float *)bd;
+        } else if (role[i] == TCPX) {
+            // GEMM row = P stored pixels; its K window is those and the next two pixels, for each
+            // of the three rows ky: steps of 32 bytes, the last one or two from the GEMM row after.
+            const int PW = slot_pw(d.in_w), G = PW / P, row = P * d.in_c;
+            const int first_ks = row / 32, n_ks = (P + 2) * d.in_c / 32;
+            g.chunk_bytes = row;
+            g.kstep_list = 1;
+            g.n_chunks = 3 * n_ks;
+            g.rows_per_image = (d.in_h + 2) * G;
+            g.grid_w = G;
+            g.shifted = 1;
+            g.a_rows = round_up(128 + 2 * G + 2, 8);
+            g.px_per_row = P;
+            g.px_cols = d.out_c;
+            g.px_w = d.in_w;
+            packed.assign((size_t)g.n_chunks * n_total * 32, 0);
+            for (int ky = 0; ky < 3; ++ky)
+                for (int ks = 0; ks < n_ks; ++ks) {
+                    const int j = ky * n_ks + ks;
+                    g.row_off[j] = ky * G + (ks < first_ks ? 0 : 1);
+                    g.col_off[j] = 32 * (ks < first_ks ? ks : ks - first_ks);
+                    for (int px = 0; px < P; ++px)
+                        for (int oc = 0; oc < d.out_c; ++oc)
+                            for (int kk = 0; kk < 32; ++kk) {
+                                const int wb = 32 * ks + kk, pin = wb / d.in_c, c = wb % d.in_c;
+                                const int kx = pin - px;
+                                if (kx < 0 || kx > 2) continue;
+                                packed[((size_t)j * n_total + px * d.out_c + oc) * 32 + kk] =
+                                    d.w[((oc * d.in_c + c) * 3 + ky) * 3 + kx];
+                            }
+                }
+            const bool relu_in = (d.flags & ACCERL_RELU_IN) && !(layers[i - 1].flags & ACCERL_RELU_OUT);
+            a_ptr = relu_in ? fin.p_slot_relu : fin.p_slot;
+            a_rows_total = (long long)p->max_batch * (d.in_h + 2) * G;
+            row_bytes = row;
+            // per-column scales and residual multipliers: the channel's, repeated for the P pixels
+            std::vector<float> ks(n_total), bs(n_total);
+            std::vector<int32_t> sm(n_total, 0);
+            for (int px = 0; px < P; ++px)
+                for (int oc = 0; oc < d.out_c; ++oc) {
+                    volatile float k = d.s_in * d.s_w[oc];
+                    ks[px * d.out_c + oc] = k;
+                    bs[px * d.out_c + oc] = d.bias[oc];
+                    if (d.skip_from >= 0) sm[px * d.out_c + oc] = d.skip_mul[oc];
+                }
+            void *kd = nullptr, *bd = nullptr, *sd = nullptr;
+            if ((st = upload_bytes(p, ks.data(), ks.size() * 4, &kd)) != ACCERL_OK) return st;
+            if ((st = upload_bytes(p, bs.data(), bs.size() * 4, &bd)) != ACCERL_OK) return st;
+            if ((st = upload_bytes(p, sm.data(), sm.size() * 4, &sd)) != ACCERL_OK) return st;
+            ks_dev = (const float *)kd;
+            bs_dev = (const float *)bd;
+            px_skip_mul = (const int32_t *)sd;
         } else if (role[i] == TCCONV) {
             const int Hp = d.in_h + 2, Wp = d.in_w + 2;
             g.chunk_bytes = 32;
@@ -452,22 +589,30 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         // outputs: every stored form of tensor i
         struct OutSpec {
             int8_t *ptr;
-            int rpi, gw, off, pitch, relu;
-        } outs[2];
+            int rpi, gw, off, pitch, relu, xmul;
+        } outs[4];
         int n_out = 0;
         if (role[i] == TCFIRST) {
-            outs[n_out++] = OutSpec{first_out, L.out_h * OW8, OW8, 0, n_total, 0};
+            outs[n_out++] = OutSpec{first_out, L.out_h * OW8, OW8, 0, n_total, 0, 1};
             TapDesc &td = p->taps[i + 1];
             td.ptr = first_out;
             td.pitch = d.out_c;
             td.hpitch = L.out_h;
             td.wpitch = OW8 * 8;
         } else if (!logits) {
-            const int H = L.out_h, W = L.out_w;
-            if (fout.plain) outs[n_out++] = OutSpec{fout.p_plain, H * W, W, 0, n_total, 0};
-            if (fout.plain_relu) outs[n_out++] = OutSpec{fout.p_plain_relu, H * W, W, 0, n_total, 1};
-            if (fout.pad || fout.pad_relu)
-                outs[n_out++] = OutSpec{fout.p_pad, (H + 2) * (W + 2), W + 2, W + 3, 32, fout.pad_relu ? 1 : 0};
+            // Row pitch = one pixel of the stored form; a multi-pixel GEMM row starts at pixel
+            // X * P and its columns run on over the following pixels.
+            const int H = L.out_h, W = L.out_w, xm = P ? P : 1, px = P ? d.out_c : n_total;
+            const int SW = slot_pw(W);
+            if (fout.plain) outs[n_out++] = OutSpec{fout.p_plain, H * W, W, 0, px, 0, xm};
+            if (fout.plain_relu) outs[n_out++] = OutSpec{fout.p_plain_relu, H * W, W, 0, px, 1, xm};
+            if (fout.pad || fout.pad_relu) {
+                if (P && d.out_c != 32) return bail();
+                outs[n_out++] = OutSpec{fout.p_pad, (H + 2) * (W + 2), W + 2, W + 3, 32, fout.pad_relu ? 1 : 0, xm};
+            }
+            if (fout.slot) outs[n_out++] = OutSpec{fout.p_slot, (H + 2) * SW, SW, SW + 1, L.out_cp, 0, xm};
+            if (fout.slot_relu)
+                outs[n_out++] = OutSpec{fout.p_slot_relu, (H + 2) * SW, SW, SW + 1, L.out_cp, 1, xm};
         }
         if (!logits) {
             if (n_out == 0 || n_out > 2) return bail();
@@ -477,6 +622,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             g.out_row_off = outs[0].off;
             g.out_pitch = outs[0].pitch;
             g.out_relu = outs[0].relu;
+            g.out_xmul = outs[0].xmul;
             if (n_out == 2) {
                 g.out2 = outs[1].ptr;
                 g.out2_rows_per_image = outs[1].rpi;
@@ -484,16 +630,29 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                 g.out2_row_off = outs[1].off;
                 g.out2_pitch = outs[1].pitch;
                 g.out2_relu = outs[1].relu;
+                g.out2_xmul = outs[1].xmul;
             }
         }
         if (d.skip_from >= 0) {
-            g.skip = forms[d.skip_from + 1].p_plain;
-            g.skip_mul = L.skip_mul;
+            const Forms &fs = forms[d.skip_from + 1];
             g.skip_pitch = p->layers[d.skip_from].out_cp;
-            g.skip_rows_per_image = L.out_h * L.out_w;
-            g.skip_grid_w = L.out_w;
-            g.skip_xmul = 1;
-            g.skip_row_off = 0;
+            if (P) {
+                const int SW = slot_pw(L.out_w);
+                g.skip = fs.p_slot;
+                g.skip_mul = px_skip_mul;
+                g.skip_rows_per_image = (L.out_h + 2) * SW;
+                g.skip_grid_w = SW;
+                g.skip_xmul = P;
+                g.skip_row_off = SW + 1;
+            } else {
+                g.skip = fs.p_plain;
+                g.skip_mul = L.skip_mul;
+                g.skip_rows_per_image = L.out_h * L.out_w;
+                g.skip_grid_w = L.out_w;
+                g.skip_xmul = 1;
+                g.skip_row_off = 0;
+            }
+            if (!g.skip) return bail();
         }
         g.kscale = ks_dev;
         g.bias = bs_dev;
@@ -515,11 +674,16 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             g.fast_div = ok ? 1 : 0;
         }
         g.split_cols = g.n_tile > 128 ? 1 : 0;
+        if (role[i] == TCPX && !g.fast_div) return bail();  // multi-pixel rows need the verified division
+        // layers that also read a residual or write a second form: collect the rows in shared memory
+        // and move whole 128-byte lines (the load/store path bounds them otherwise)
+        g.staged = (role[i] == TCPX && g.n_tile == 128 && (g.skip || g.out2)) ? 1 : 0;
         g.logits_mode = logits ? 1 : 0;
         g.n_actions = p->n_actions;
         g.status = p->status_word;
         g.trace_slot = (int)p->tc_steps.size() % 8;
-        ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * g.chunk_bytes <= 96 * 1024;
+        const int b_bytes = g.kstep_list ? 32 : g.chunk_bytes;  // bytes of a weight row per chunk
+        ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * b_bytes <= 96 * 1024;
         if (g.shifted && !ts.resident_b) return bail();
         if (!tc_choose_pipeline(g, ts.resident_b)) {
             if (g.shifted) return bail();
@@ -531,8 +695,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if ((st = tc_make_map(ts.map_a, a_ptr, a_rows_total, row_bytes, row_bytes,
                               g.shifted ? g.a_rows : 128, g.chunk_bytes)) != ACCERL_OK)
             return st;
-        if ((st = tc_make_map(ts.map_b, w_dev, (long long)g.n_chunks * n_total, g.chunk_bytes,
-                              g.chunk_bytes, g.n_tile, g.chunk_bytes)) != ACCERL_OK)
+        if ((st = tc_make_map(ts.map_b, w_dev, (long long)g.n_chunks * n_total, b_bytes, b_bytes, g.n_tile,
+                              b_bytes)) != ACCERL_OK)
             return st;
         p->tc_steps.push_back(ts);
         s.kind = Step::TC_GEMM;
