@@ -486,6 +486,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = bars.tmem_base;
+    // Programmatic dependent launch: the next tensor-core launch may start its own set-up (barriers,
+    // tensor memory, weights) on SMs this grid has left; it waits for this grid's completion before
+    // it touches activations (griddepcontrol.wait in the producer and epilogue roles).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int total_tiles = ((p.m_tiles + SUB - 1) / SUB) * p.n_tiles;  // pipeline steps
 #ifdef ACCERL_TC_TRACE
@@ -522,6 +526,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             __syncwarp();
         }
+        // the activations are the previous launch's output
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         bool ok = true;
         int base_slot = 0;  // ring position of the current tile inside this warp's ring
         uint32_t base_phase = 0;
@@ -664,6 +670,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         c.s_skip_mul = s_skip_mul;
         c.abort_flag = abort_flag;
         c.staging = stages + (size_t)n_stages * stage_bytes;
+        // outputs may reuse buffers that the previous launch still reads
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         if constexpr (PXK) {  // multi-pixel rows: only built for the verified division
             if (p.staged) {
                 if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, true>(p, c, warp, lane);
@@ -816,8 +824,17 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        kernel<<<grid, kThreads, smem, st>>>(*(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, p);
-        return cudaSuccess;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, p);
     };
     cudaError_t e;
     if (p.px_per_row) {
