@@ -296,13 +296,17 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
         case Step::INGEST_NHWC4:
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut,
                                                    p->bufs[p->layers[0].in_buf].ptr, B, p->in_h,
-                                                   p->in_w, p->in_h, p->in_w, 0, 0, p->ingest_arith,
-                                                   p->ingest_mul, p->ingest_add, st));
+                                                   p->in_w, p->in_h, p->in_w, 0, 0,
+                                                   p->ingest_float ? 2 : p->ingest_arith,
+                                                   p->ingest_float ? p->ingest_fa : p->ingest_mul,
+                                                   p->ingest_float ? p->ingest_fc1 : p->ingest_add, st));
             break;
         case Step::INGEST_PAD4:
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut, p->in_pad4, B,
                                                    p->in_h, p->in_w, p->in_h + 2, p->in_pad4_w, 1, 4,
-                                                   p->ingest_arith, p->ingest_mul, p->ingest_add, st));
+                                                   p->ingest_float ? 2 : p->ingest_arith,
+                                                   p->ingest_float ? p->ingest_fa : p->ingest_mul,
+                                                   p->ingest_float ? p->ingest_fc1 : p->ingest_add, st));
             break;
         case Step::POOL_DUAL:
             ACCERL_CUDA_TRY(launch_maxpool_dual(p->pools[s.tc], B, st));
@@ -526,6 +530,10 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         }
         if ((st = upload(p, lut, &p->lut)) != ACCERL_OK) return fail(st);
         p->ingest_arith = fit_ingest_line(lut.data(), &p->ingest_mul, &p->ingest_add) ? 1 : 0;
+        // the float form of the line (measured faster in the NHWC kernel, slower in the space-to-depth one)
+        p->ingest_float = p->ingest_arith == 1 &&
+                          fit_ingest_float_line(lut.data(), p->ingest_mul, p->ingest_add, &p->ingest_fa,
+                                                &p->ingest_fc1);
     }
     {
         std::vector<int> zero(256, 0);  // word 0 is the status; the rest is trace space

@@ -43,6 +43,7 @@ __device__ __forceinline__ int8_t requant(float y, float s_out)
 // otherwise the element is redone with the exact divide.  Saturating conversion and saturating
 // packing implement the clamp to [-128, 127].
 constexpr float kTieGuard = 4e-5f;
+constexpr float kRoundMagic = 12582912.f;  // 1.5 * 2^23: adding it rounds to the nearest integer
 
 __device__ __forceinline__ uint32_t pack4_sat_s8(int a0, int a1, int a2, int a3)
 {
@@ -132,6 +133,27 @@ __device__ __forceinline__ void requant16_fastdiv(const int (&acc)[16], const fl
     }
 #pragma unroll
     for (int g = 0; g < 4; ++g) w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
+}
+
+// Four frame bytes (byte `dx` of the words p0..p3, one per channel plane) -> four int8 codes in one
+// word, channel 0 in the low byte, without integer multiplies: a byte permute builds the float
+// 128 + u/256 from byte u, two packed float operations map it onto 1.5 * 2^23 + code (rounded to
+// nearest by the addition itself), and the codes are the low bytes of the bit patterns.  The two
+// constants come from fit_ingest_float_line(), which has checked all 256 inputs on the host.
+__device__ __forceinline__ uint32_t ingest_float_line4(uint32_t p0, uint32_t p1, uint32_t p2, uint32_t p3,
+                                                       int dx, float A, float c1)
+{
+    const uint32_t sel = 0x7404u | ((uint32_t)dx << 4);  // bytes: 00, u, 00, 0x43
+    const float2 f01 = make_float2(__uint_as_float(__byte_perm(p0, 0x43000000u, sel)),
+                                   __uint_as_float(__byte_perm(p1, 0x43000000u, sel)));
+    const float2 f23 = make_float2(__uint_as_float(__byte_perm(p2, 0x43000000u, sel)),
+                                   __uint_as_float(__byte_perm(p3, 0x43000000u, sel)));
+    const float2 nc = make_float2(-c1, -c1), a2 = make_float2(A, A), mg = make_float2(kRoundMagic, kRoundMagic);
+    const float2 r01 = __ffma2_rn(__fadd2_rn(f01, nc), a2, mg);
+    const float2 r23 = __ffma2_rn(__fadd2_rn(f23, nc), a2, mg);
+    const uint32_t lo = __byte_perm(__float_as_uint(r01.x), __float_as_uint(r01.y), 0x0040);
+    const uint32_t hi = __byte_perm(__float_as_uint(r23.x), __float_as_uint(r23.y), 0x0040);
+    return __byte_perm(lo, hi, 0x5410);
 }
 
 }  // namespace accerl

@@ -22,6 +22,7 @@
 
 #include <algorithm>
 
+#include "epilogue.cuh"
 #include "internal.h"
 
 namespace accerl {
@@ -86,7 +87,7 @@ cudaError_t launch_maxpool_dual(const PoolDualParams &q, int B, cudaStream_t st)
 // ---------------------------------------------------------------------------------------
 // uint8 NCHW frames with 4 channels -> plain int8 NHWC: four pixels per thread
 // ---------------------------------------------------------------------------------------
-template <bool ARITH>
+template <int ARITH>
 __global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const int8_t *__restrict__ lut,
                                        int8_t *__restrict__ out, long long total, int H, int W4,
                                        int out_hpitch, int out_wpitch, int off_y, int off_x,
@@ -112,7 +113,10 @@ __global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const in
     uint32_t w[4];
 #pragma unroll
     for (int px = 0; px < 4; ++px) {
-        if (ARITH) {
+        if (ARITH == 2) {
+            w[px] = ingest_float_line4(plane[0], plane[1], plane[2], plane[3], px, __uint_as_float(mul),
+                                       __uint_as_float(add));
+        } else if (ARITH == 1) {
             uint32_t pr[4];
 #pragma unroll
             for (int c = 0; c < 4; ++c) pr[c] = ((plane[c] >> (8 * px)) & 0xff) * mul + add;
@@ -137,12 +141,15 @@ cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t
 {
     const long long total = (long long)B * H * (W / 4);
     const unsigned blocks = (unsigned)((total + 255) / 256);
-    if (arith)
-        ingest_u8_nhwc4_kernel<true><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
-                                                            out_wpitch, off_y, off_x, mul, add);
+    if (arith == 2)
+        ingest_u8_nhwc4_kernel<2><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
+                                                         out_wpitch, off_y, off_x, mul, add);
+    else if (arith == 1)
+        ingest_u8_nhwc4_kernel<1><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
+                                                         out_wpitch, off_y, off_x, mul, add);
     else
-        ingest_u8_nhwc4_kernel<false><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
-                                                             out_wpitch, off_y, off_x, mul, add);
+        ingest_u8_nhwc4_kernel<0><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
+                                                         out_wpitch, off_y, off_x, mul, add);
     return cudaGetLastError();
 }
 

@@ -18,38 +18,43 @@ namespace accerl {
 // line that the host has checked against all 256 table entries; the product fits 32 bits, so the
 // code is simply the top byte of the multiply-add.
 // ---------------------------------------------------------------------------------------
-template <bool ARITH>
+template <int ARITH>
 __global__ void ingest_u8_s2d44_kernel(const uint8_t *__restrict__ obs,
                                        const int8_t *__restrict__ lut, uint4 *__restrict__ out,
-                                       long long total, int H, int W, uint32_t mul, uint32_t add)
+                                       int B, int H, int W, uint32_t mul, uint32_t add)
 {
     __shared__ int8_t s_lut[256];
     if (!ARITH) {
         for (int i = threadIdx.x; i < 256; i += blockDim.x) s_lut[i] = lut[i];
         __syncthreads();
     }
-    long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= total) return;
-    const int Ws = W / 4, Hs = H / 4;
-    // one thread = one output row (n, Y, X): sixteen independent 4-byte loads (4 image rows of 4
-    // channel planes) are in flight before the first is used, then 64 contiguous bytes are stored
-    int X = (int)(idx % Ws);
-    long long t = idx / Ws;
-    int Y = (int)(t % Hs);
-    long long n = t / Hs;
+    // One block = one image, one thread = one output row (Y, X); all index arithmetic is 32-bit
+    // and per image (the kernel is bound by integer instructions, not by memory).  Sixteen
+    // independent 4-byte loads (4 image rows of 4 channel planes) are in flight before the first
+    // is used, then 64 contiguous bytes are stored.
+    const int Ws = W / 4, rows = (H / 4) * Ws;
+    const int pos = blockIdx.y * blockDim.x + threadIdx.x;
+    if (pos >= rows) return;
+    const int n = blockIdx.x;
+    const int Y = pos / Ws, X = pos - Y * Ws;
+    const uint8_t *img = obs + (size_t)n * 4 * H * W + (4 * Y) * W + 4 * X;
+    const long long idx = (long long)n * rows + pos;
+    const int plane_bytes = H * W;
     uint32_t plane[4][4];  // [dy][c]
 #pragma unroll
     for (int dy = 0; dy < 4; ++dy)
 #pragma unroll
         for (int c = 0; c < 4; ++c)
-            plane[dy][c] = __ldg(reinterpret_cast<const uint32_t *>(
-                obs + ((n * 4 + c) * H + 4 * Y + dy) * W + 4 * X));
+            plane[dy][c] = __ldg(reinterpret_cast<const uint32_t *>(img + c * plane_bytes + dy * W));
 #pragma unroll
     for (int dy = 0; dy < 4; ++dy) {
         uint32_t w[4];
 #pragma unroll
         for (int dx = 0; dx < 4; ++dx) {
-            if (ARITH) {
+            if (ARITH == 2) {
+                w[dx] = ingest_float_line4(plane[dy][0], plane[dy][1], plane[dy][2], plane[dy][3], dx,
+                                           __uint_as_float(mul), __uint_as_float(add));
+            } else if (ARITH == 1) {
                 uint32_t pr[4];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) pr[c] = ((plane[dy][c] >> (8 * dx)) & 0xff) * mul + add;
@@ -128,19 +133,51 @@ bool fit_ingest_line(const int8_t *lut, uint32_t *mul, uint32_t *add)
     return false;
 }
 
+// The same table as a float line (see ingest_float_line4 in epilogue.cuh): byte u becomes the float
+// 128 + u/256 by a byte permute, g = that - c1, r = fma(g, A, 1.5 * 2^23), and the code is the low
+// byte of r's bit pattern.  Starting from the fixed-point line, a few offsets are tried and each
+// candidate is run through exactly the device's float operations for all 256 inputs.
+bool fit_ingest_float_line(const int8_t *lut, uint32_t mul, uint32_t add, uint32_t *a_bits, uint32_t *c1_bits)
+{
+    const double one = 16777216.0, m = (double)mul / one;
+    for (int i = 0; i < 256; ++i)
+        if (lut[i] < 0) return false;
+    for (int t = -8; t <= 8; ++t) {
+        const double k = (double)add / one - 0.5 + t * 2.5e-4;  // floor(x) = rint(x - 1/2) off the ties
+        const float A = (float)(256.0 * m);
+        const float c1 = (float)(128.0 - k / (double)A);
+        bool ok = true;
+        for (int u = 0; u < 256 && ok; ++u) {
+            uint32_t fb = 0x43000000u | ((uint32_t)u << 8), rb;
+            float f, r;
+            memcpy(&f, &fb, 4);
+            volatile float g = f - c1;
+            r = fmaf(g, A, 12582912.0f);
+            memcpy(&rb, &r, 4);
+            ok = (rb & 0xffu) == (uint32_t)lut[u] && r >= 12582912.0f && r < 12582912.0f + 128.0f;
+        }
+        if (ok) {
+            memcpy(a_bits, &A, 4);
+            memcpy(c1_bits, &c1, 4);
+            return true;
+        }
+    }
+    return false;
+}
+
 cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *out, int B, int C,
                                  int H, int W, int s, int arith, uint32_t mul, uint32_t add,
                                  cudaStream_t st)
 {
     if (C == 4 && s == 4 && W % 4 == 0) {
-        long long total = (long long)B * (H / 4) * (W / 4);
-        const unsigned blocks = (unsigned)((total + 255) / 256);
-        if (arith)
-            ingest_u8_s2d44_kernel<true><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, H, W,
-                                                                mul, add);
+        const int rows = (H / 4) * (W / 4), threads = rows >= 448 ? 224 : 128;
+        const dim3 grid((unsigned)B, (unsigned)((rows + threads - 1) / threads));
+        if (arith == 2)
+            ingest_u8_s2d44_kernel<2><<<grid, threads, 0, st>>>(obs, lut, (uint4 *)out, B, H, W, mul, add);
+        else if (arith == 1)
+            ingest_u8_s2d44_kernel<1><<<grid, threads, 0, st>>>(obs, lut, (uint4 *)out, B, H, W, mul, add);
         else
-            ingest_u8_s2d44_kernel<false><<<blocks, 256, 0, st>>>(obs, lut, (uint4 *)out, total, H, W,
-                                                                 mul, add);
+            ingest_u8_s2d44_kernel<0><<<grid, threads, 0, st>>>(obs, lut, (uint4 *)out, B, H, W, mul, add);
     } else {
         long long total = (long long)B * C * H * W;
         ingest_u8_s2d_any_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(obs, lut, out, total,
