@@ -103,6 +103,13 @@ def algorithmic(name: str, batch: int) -> dict:
                 bytes=(W.input_bytes_per_state(name) + 4 + OUT_BYTES(a)) * batch)
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch / states of that launch, from
+# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 188.85 MB read + 127.19 MB written)
+NCU_DRAM_BYTES_PER_STATE = {
+    ("nature_cnn_b8192", "ingest_u8_s2d44_kernel"): (188851968 + 127191040) / 6144,
+}
+
+
 def launch_work(name: str, plan: str, batch: int) -> list:
     """Per launch of the plan: kernel name, int8 ops (2 x MACs) and algorithmic bytes."""
     c = W.config(name)
@@ -328,7 +335,11 @@ def main() -> None:
         achieved = work[top]["bytes"] / (per[top] * 1e-3) / 1e9
         roof = dict(bound="hbm", achieved=achieved, peak=pk["hbm_gbs"], unit="GB/s",
                     frac=achieved / pk["hbm_gbs"])
-    roof.update(traffic=None, kernel=work[top]["kernel"], covers=work[top]["covers"],
+    # DRAM bytes per launch from the committed ncu capture of this kernel (profiles/), measured on
+    # a smaller batch and scaled by the states processed; None for kernels without a capture
+    per_state = NCU_DRAM_BYTES_PER_STATE.get((name, work[top]["kernel"]))
+    traffic = None if per_state is None else per_state * batch
+    roof.update(traffic=traffic, kernel=work[top]["kernel"], covers=work[top]["covers"],
                 kernel_ms=float(per[top]), share=float(per[top] / per.sum()),
                 peak_source="%s (int8 = 2 x bf16 burst)" % pk["source"] if roof["bound"] == "tensor"
                 else pk["source"])
