@@ -228,7 +228,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                               ((d.flags & ACCERL_LOGITS) ? d.out_c <= 256
                                                          : (d.out_c % 16 == 0 && d.out_c <= kTcMaxN &&
                                                             (d.out_c <= 256 || d.out_c % 256 == 0)));
-            if (!fits) return ACCERL_OK;
+            if (!fits && !fc_sample_fits(p, layers, n_layers, i)) return ACCERL_OK;
             role[i] = TCFC;
         } else if (d.kind == ACCERL_CONV2D && d.skip_from < 0 && i == 0) {
             // A first conv on 4-channel frames: tensor cores if its only reader is a max-pool (see
@@ -288,7 +288,6 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         if (f.count() > 2) return ACCERL_OK;
         if (t > 0 && (role[t - 1] == GENERIC || role[t - 1] == TCFIRST) && (f.count() != 1 || !f.plain))
             return ACCERL_OK;
-        if (t > 0 && role[t - 1] == POOL && f.plain_relu) return ACCERL_OK;
         if (t > 0 && role[t - 1] == TCPX && (f.pad || f.pad_relu) && layers[t - 1].out_c != 32)
             return ACCERL_OK;
     }
@@ -404,8 +403,10 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             int n_po = 0;
             const int OH = L.out_h, OW = L.out_w, C = L.in_c;
             if (fout.plain) q.out[n_po++] = PoolOut{fout.p_plain, OH, OW, 0, 0, C, 0};
-            if (fout.pad || fout.pad_relu)
+            if (fout.plain_relu) q.out[n_po++] = PoolOut{fout.p_plain_relu, OH, OW, 0, 0, C, 1};
+            if ((fout.pad || fout.pad_relu) && n_po < 2)
                 q.out[n_po++] = PoolOut{fout.p_pad, OH + 2, OW + 2, 1, 1, 32, fout.pad_relu ? 1 : 0};
+            else if (fout.pad || fout.pad_relu) return bail();
             if (fout.slot && n_po < 2) q.out[n_po++] = PoolOut{fout.p_slot, OH + 2, slot_pw(OW), 1, 1, C, 0};
             else if (fout.slot) return bail();
             if (fout.slot_relu && n_po < 2)

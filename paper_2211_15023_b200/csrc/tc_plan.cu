@@ -273,6 +273,8 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         if ((d.flags & ACCERL_RELU_IN) && !relu_in_noop) return ACCERL_OK;
         if (d.kind == ACCERL_CONV2D) {
             if (!conv_fits(d)) return ACCERL_OK;
+        } else if (d.kind == ACCERL_FC && fc_sample_fits(p, layers, n_layers, i)) {
+            // runs fused with the sampler, whatever its size
         } else if (d.kind == ACCERL_FC) {
             const int K = L.in_h * L.in_w * L.in_cp;
             if (L.in_cp != L.in_c || K % 16 || K < 128 || (K + 127) / 128 > kTcMaxChunks)

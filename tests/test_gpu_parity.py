@@ -161,6 +161,44 @@ def test_odd_shapes_padding_stride_pool_residual():
     g.close()
 
 
+@pytest.mark.parametrize("hw", [(44, 40), (37, 52)], ids=["19_wide_after_pool", "25_wide_after_pool"])
+def test_multi_pixel_rows_ragged_widths(hw):
+    """Residual 3x3 stacks on images whose width is no multiple of the pixels per GEMM row: the
+    last group of a row is cut (19 = 2*8+3, 25 = 3*8+1; the 16->32 conv and the 32-channel block
+    use 4 pixels per row), with and without taps, so that both the direct and the shared-memory
+    staged epilogues, the residual read and the ReLU'd second copy are compared with the oracle."""
+    import paper_2211_15023_b200 as P
+    H, Wd = hw
+    rng = np.random.default_rng(23)
+    h1, w1 = (H - 3) // 2 + 1, (Wd - 3) // 2 + 1
+    layers = [W._conv(4, H, Wd, 16, 3, 1, 1, relu_out=False), W._pool(16, H, Wd),
+              W._conv(16, h1, w1, 16, 3, 1, 1, relu_in=True, relu_out=True),
+              W._conv(16, h1, w1, 16, 3, 1, 1, relu_out=False, skip_from=1),
+              W._conv(16, h1, w1, 32, 3, 1, 1, relu_out=False),
+              W._conv(32, h1, w1, 32, 3, 1, 1, relu_in=True, relu_out=True),
+              W._conv(32, h1, w1, 32, 3, 1, 1, relu_out=False, skip_from=4),
+              W._pool(32, h1, w1)]
+    h2, w2 = (h1 - 3) // 2 + 1, (w1 - 3) // 2 + 1
+    layers += [W._fc(32 * h2 * w2, 64, relu_in=True), W._fc(64, 6, relu_out=False, logits=True)]
+    params = [None if l["kind"] == "maxpool" else
+              dict(w=(rng.standard_normal((l["out_c"], l["in_c"], l["kh"], l["kw"])) *
+                      np.sqrt(2.0 / (l["in_c"] * l["kh"] * l["kw"]))).astype(np.float32),
+                   bias=rng.standard_normal(l["out_c"]).astype(np.float32) * 0.05) for l in layers]
+    calib = rng.integers(0, 256, (32, 4, H, Wd), dtype=np.uint8)
+    pol = oracle.calibrate("u8", (4, H, Wd), layers, params, calib)
+    b = 11
+    obs = rng.integers(0, 256, (b, 4, H, Wd), dtype=np.uint8)
+    u = rng.random(b, dtype=np.float32)
+    ref = oracle.forward(pol, obs, u)
+    for flags in (1, 0):
+        g = P.Policy(pol, b, flags=flags)
+        assert "tc_gemm_kernel" in g.info()["plan"]
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        g.check()
+        compare(ref, *out, taps=g.read_activation if flags else None)
+        g.close()
+
+
 def test_exact_ties_on_the_tensor_core_path():
     """Power-of-two scales make many epilogue quotients land exactly on k + 0.5: the requantiser
     must round them to even exactly as the IEEE divide + rintf of the definition does."""
