@@ -821,6 +821,12 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
     const int tiles = ((p.m_tiles + p.sub - 1) / p.sub) * p.n_tiles;
     const int grid = tiles < sm_count ? tiles : sm_count;
     const bool extras = p.skip || p.out2 || p.out_relu || p.out2_relu;
+    // One tile per CTA at most (a fully connected layer at these batch sizes): a single issuing warp
+    // then owns every shared-memory stage instead of its share of them, which doubles or
+    // quadruples how far the loads run ahead of the MMAs.
+    TcGemmParams one = p;
+    if (!p.shifted && p.sub == 1 && tiles <= sm_count) one.n_mma = 1;
+    const TcGemmParams &q = one;
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -834,7 +840,7 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, p);
+        return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, q);
     };
     cudaError_t e;
     if (p.px_per_row) {
