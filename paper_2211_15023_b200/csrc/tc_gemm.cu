@@ -190,6 +190,7 @@ struct __align__(8) Barriers {
 struct EpiCtx {
     uint32_t tmem_base, acc_full0, acc_empty0;
     int total_tiles, n_acc, acc_stride, acc_cols, sub;
+    int parts, sets_log2;  // K-split: partial accumulators per tile, log2 of the accumulator sets
     const float *s_ks, *s_bs;
     const int *s_skip_mul;
     volatile int *abort_flag;
@@ -224,7 +225,7 @@ __device__ __forceinline__ uint4 relu_codes(uint4 v)
 // instruction, and the load/store path then bounds the layer.  Instead every warp collects its 32
 // rows in a shared-memory tile and copies it out with eight lanes per row, full lines per
 // instruction; the residual source comes in the same way.
-template <bool EXTRAS, int MODE, bool RELU, bool PX, bool STAGED>
+template <bool EXTRAS, int MODE, bool RELU, bool PX, bool STAGED, bool KS>
 __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
 {
     uint8_t *stage = STAGED ? c.staging + (warp - kProdWarps - kMmaWarps) * kStagingBytes : nullptr;
@@ -244,8 +245,9 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
             mt = t / p.n_tiles;
             nt = t - mt * p.n_tiles;
         }
-        const int a = tile_i & (c.n_acc - 1);  // n_acc is a power of two
-        const uint32_t apar = (tile_i >> p.n_acc_log2) & 1;
+        // accumulator stage (n_acc is a power of two); with K-split the first of the tile's partials
+        const int a = (KS && c.parts > 1) ? (tile_i & ((1 << c.sets_log2) - 1)) * c.parts : tile_i & (c.n_acc - 1);
+        const uint32_t apar = (tile_i >> ((KS && c.parts > 1) ? c.sets_log2 : p.n_acc_log2)) & 1;
         {
             TRACE_T0();
             ok = mbar_wait(c.acc_full0 + 8 * a, apar, c.abort_flag, p.status, 16);
@@ -322,6 +324,13 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                     TRACE_T0();
                     tmem_ld16(taddr + c0, acc);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    for (int part = 1; KS && part < c.parts; ++part) {  // K-split: add the other partial sums
+                        int more[16];
+                        tmem_ld16(taddr + part * c.acc_stride + c0, more);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[i] += more[i];
+                    }
                     if (threadIdx.x == 32 * (kProdWarps + kMmaWarps)) TRACE_ADD(7);
                 }
                 if (c0 + 16 >= c_end && sub == c.sub - 1) {
@@ -430,6 +439,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // K-split is only compiled into the kernels with streamed weights (fully connected layers)
+    constexpr bool KS = !RESIDENT_B;
+    const bool ksplit = KS && p.ksplit;
     const int CH = p.chunk_bytes;
     const int a_chunk_bytes = kTileM * CH;
     const int CHB = p.kstep_list ? 32 : CH;  // bytes of a weight row per chunk
@@ -468,7 +480,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(smem_u32(&bars.empty[s]), 1);
         }
         for (int a = 0; a < n_acc; ++a) {
-            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_full[a]), (!RESIDENT_B && p.ksplit) ? p.n_mma : 1);
             mbar_init(smem_u32(&bars.acc_empty[a]), p.split_cols ? 4 * kEpiGroups : 4);
         }
         mbar_init(smem_u32(&bars.b_ready), 1);
@@ -532,16 +544,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int base_slot = 0;  // ring position of the current tile inside this warp's ring
         uint32_t base_phase = 0;
         int t = blockIdx.x + pw * gridDim.x;
-        for (int i = pw; i < my_tiles && ok && pw < n_mma; i += n_mma, t += n_mma * gridDim.x) {
+        // K-split: every warp serves every tile, with the K groups pw, pw + n_mma, ...
+        const int tile_step = ksplit ? 1 : n_mma, g_first = ksplit ? pw : 0, g_step = ksplit ? n_mma : 1;
+        const int my_groups = g_first < n_groups ? (n_groups - g_first + g_step - 1) / g_step : 0;
+        if (ksplit) t = blockIdx.x;
+        for (int i = ksplit ? 0 : pw; i < my_tiles && ok && pw < n_mma; i += tile_step, t += tile_step * gridDim.x) {
             int mt = t, nt = 0;
             if (p.n_tiles != 1) {
                 mt = t / p.n_tiles;
                 nt = t - mt * p.n_tiles;
             }
             const int row0 = mt * kTileM * SUB, brow0 = nt * p.n_tile;
-            for (int gi = 0; gi < n_groups; ++gi) {
+            for (int gq = 0; gq < my_groups; ++gq) {
+                const int gi = g_first + gq * g_step;
                 const int j = gi * G;
-                int sl = base_slot + gi;
+                int sl = base_slot + gq;
                 uint32_t ph = base_phase;
                 while (sl >= ring) {
                     sl -= ring;
@@ -575,7 +592,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 __syncwarp();
             }
-            base_slot += n_groups;
+            base_slot += my_groups;
             while (base_slot >= ring) {
                 base_slot -= ring;
                 base_phase ^= 1;
@@ -599,18 +616,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (RESIDENT_B) ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
         int a = mw, base_slot = 0;
         uint32_t aphase = 0, base_phase = 0;
-        for (int i = mw; i < my_tiles && ok && mw < n_mma; i += n_mma) {
+        const int tile_step = ksplit ? 1 : n_mma, g_first = ksplit ? mw : 0, g_step = ksplit ? n_mma : 1;
+        const int my_groups = g_first < n_groups ? (n_groups - g_first + g_step - 1) / g_step : 0;
+        for (int i = ksplit ? 0 : mw; i < my_tiles && ok && mw < n_mma; i += tile_step) {
             const uint32_t apar = aphase ^ 1;
+            // K-split: the barriers of a tile are those of its first partial accumulator
+            const int a_bar = ksplit ? a - mw : a;
             {
                 TRACE_T0();
-                ok = mbar_wait(acc_empty0 + 8 * a, apar, abort_flag, p.status, 4);
+                ok = mbar_wait(acc_empty0 + 8 * a_bar, apar, abort_flag, p.status, 4);
                 TRACE_ADD(1);
             }
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t d_tmem = tmem_base + (uint32_t)(a * acc_stride);
-            for (int gi = 0; gi < n_groups; ++gi) {
-                int sl = base_slot + gi;
+            for (int gq = 0; gq < my_groups; ++gq) {
+                const int gi = g_first + gq * g_step;
+                int sl = base_slot + gq;
                 uint32_t par = base_phase;
                 while (sl >= ring) {
                     sl -= ring;
@@ -634,21 +656,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             const uint2 rel = s_desc[t];
                             const uint32_t b_lo = RESIDENT_B ? rel.y : st_lo + rel.y;
                             mma_i8(d_tmem + sub * acc_cols, desc_hi | (sub_lo + rel.x), desc_hi_b | b_lo,
-                                   idesc, (uint32_t)t);
+                                   idesc, (uint32_t)(t - g_first * G * k_steps));  // 0: first K step of this warp
                         }
                     }
                     mma_commit(empty0 + 8 * s);  // frees the stage when the MMAs retire
                 }
                 __syncwarp();
             }
-            if (ok && elect_one()) mma_commit(acc_full0 + 8 * a);
+            if (ok && elect_one()) mma_commit(acc_full0 + 8 * a_bar);
             __syncwarp();
             a += n_mma;
             if (a >= n_acc) {
                 a -= n_acc;
                 aphase ^= 1;
             }
-            base_slot += n_groups;
+            base_slot += my_groups;
             while (base_slot >= ring) {
                 base_slot -= ring;
                 base_phase ^= 1;
@@ -665,6 +687,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         c.acc_stride = acc_stride;
         c.acc_cols = acc_cols;
         c.sub = SUB;
+        c.parts = ksplit ? n_mma : 1;
+        c.sets_log2 = 0;
+        while ((n_mma << c.sets_log2) < n_acc) ++c.sets_log2;
         c.s_ks = s_ks;
         c.s_bs = s_bs;
         c.s_skip_mul = s_skip_mul;
@@ -674,20 +699,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if constexpr (PXK) {  // multi-pixel rows: only built for the verified division
             if (p.staged) {
-                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, true>(p, c, warp, lane);
-                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, true>(p, c, warp, lane);
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, true, KS>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, true, KS>(p, c, warp, lane);
             } else {
-                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, false>(p, c, warp, lane);
-                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, false>(p, c, warp, lane);
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, false, KS>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, false, KS>(p, c, warp, lane);
             }
         } else {
-            if (p.logits_mode) epilogue_role<false, kEpiLogits, false, false, false>(p, c, warp, lane);
+            if (p.logits_mode) epilogue_role<false, kEpiLogits, false, false, false, KS>(p, c, warp, lane);
             else if (p.fast_div) {
-                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, false, false>(p, c, warp, lane);
-                else epilogue_role<EXTRAS, kEpiFastDiv, false, false, false>(p, c, warp, lane);
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, false, false, KS>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiFastDiv, false, false, false, KS>(p, c, warp, lane);
             } else {
-                if (p.relu_out) epilogue_role<EXTRAS, kEpiTieCheck, true, false, false>(p, c, warp, lane);
-                else epilogue_role<EXTRAS, kEpiTieCheck, false, false, false>(p, c, warp, lane);
+                if (p.relu_out) epilogue_role<EXTRAS, kEpiTieCheck, true, false, false, KS>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kEpiTieCheck, false, false, false, KS>(p, c, warp, lane);
             }
         }
     }
@@ -807,6 +832,8 @@ bool tc_choose_pipeline(TcGemmParams &p, bool resident_b)
                 p.tmem_cols = cols;
                 p.n_acc_log2 = 0;
                 while ((1 << p.n_acc_log2) < p.n_acc_stages) ++p.n_acc_log2;
+                // long K loops outside shifted mode: the issuing warps share each tile
+                p.ksplit = (!resident_b && !p.shifted && p.n_mma >= 2 && p.n_chunks / p.group >= 2 * p.n_mma) ? 1 : 0;
                 return true;
             }
         }
@@ -825,7 +852,7 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
     // then owns every shared-memory stage instead of its share of them, which doubles or
     // quadruples how far the loads run ahead of the MMAs.
     TcGemmParams one = p;
-    if (!p.shifted && p.sub == 1 && tiles <= sm_count) one.n_mma = 1;
+    if (!p.shifted && p.sub == 1 && !p.ksplit && tiles <= sm_count) one.n_mma = 1;
     const TcGemmParams &q = one;
     auto go = [&](auto kernel) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -25,6 +25,11 @@ struct TcGemmParams {
     int n_stages, n_acc_stages, n_acc_log2, tmem_cols;
     int group;  // K chunks per shared-memory stage
     int n_mma;  // MMA-issuing warps in use
+    // ksplit = 1 (not in shifted mode): the issuing warps share every tile instead of taking tiles in
+    // turn -- warp w contracts the K groups w, w + n_mma, ... into an accumulator of its own and the
+    // epilogue adds the n_mma partial sums (a K loop of a hundred MMAs is bound by the rate at
+    // which one thread can issue them)
+    int ksplit;
     // shifted = 1: every chunk reads the same columns at a different row offset, so one TMA box of
     // a_rows = 128 + max(row_off) rows per tile serves all of them (needs resident weights)
     int shifted, a_rows;

@@ -440,6 +440,12 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         g.out_xmul = g.out2_xmul = 1;
         g.n_total = n_total;
         g.n_tile = n_total > 256 ? 256 : n_total;
+        if (d.kind == ACCERL_FC && !logits) {
+            // small batches: narrower tiles, so that the weight stream is shared by more SMs
+            const int m_tiles = (p->max_batch + 127) / 128;
+            while (g.n_tile > 32 && g.n_tile % 32 == 0 && 2 * m_tiles * (n_total / g.n_tile) <= p->sm_count)
+                g.n_tile /= 2;
+        }
         g.n_tiles = n_total / g.n_tile;
         std::vector<int8_t> packed;
         const int8_t *a_ptr;

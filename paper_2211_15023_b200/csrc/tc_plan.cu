@@ -326,6 +326,12 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         const int n_total = round_up(d.out_c, 16);
         g.n_total = n_total;
         g.n_tile = n_total > 256 ? 256 : n_total;
+        if (d.kind == ACCERL_FC && !logits) {
+            // small batches: narrower tiles, so that the weight stream is shared by more SMs
+            const int m_tiles = (p->max_batch + 127) / 128;
+            while (g.n_tile > 32 && g.n_tile % 32 == 0 && 2 * m_tiles * (n_total / g.n_tile) <= p->sm_count)
+                g.n_tile /= 2;
+        }
         g.n_tiles = n_total / g.n_tile;
         int rows_in_per_image, row_bytes;
         std::vector<int8_t> packed;
