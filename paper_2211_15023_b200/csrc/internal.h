@@ -88,6 +88,7 @@ struct PoolDualParams {
     const int8_t *in;            // pixels of C bytes
     int in_hpitch, in_wpitch, in_off_y, in_off_x;
     int H, W, C, OH, OW, k, stride;
+    int kw, stride_x;  // window width and horizontal stride (k and stride when the input is not pre-pooled)
     PoolOut out[2];
 };
 

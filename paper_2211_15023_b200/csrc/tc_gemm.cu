@@ -411,6 +411,63 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
     }
 }
 
+// Epilogue for hpool layers (see TcGemmParams::hpool): all four warpgroups share every tile,
+// warpgroup j produces pooled pixel j of each row from the accumulators of pixels 2j .. 2j+2.
+template <bool RELU>
+__device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
+{
+    const int q = warp & 3, wg = (warp - kProdWarps - kMmaWarps) >> 2;
+    const float s_out = p.s_out, inv_s_out = p.inv_s_out;
+    int tile_i = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < c.total_tiles && ok; t += gridDim.x, ++tile_i) {
+        const int a = tile_i & (c.n_acc - 1);
+        const uint32_t apar = (tile_i >> p.n_acc_log2) & 1;
+        ok = mbar_wait(c.acc_full0 + 8 * a, apar, c.abort_flag, p.status, 16);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int m = t * kTileM + q * 32 + lane;
+        int n = __float2int_rz(__int2float_rn(m) * p.inv_rows_per_image);
+        int r = m - n * p.rows_per_image;
+        while (r < 0) {
+            --n;
+            r += p.rows_per_image;
+        }
+        while (r >= p.rows_per_image) {
+            ++n;
+            r -= p.rows_per_image;
+        }
+        const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
+        const int pc = X * 4 + wg;  // pooled column
+        const bool valid = n < p.batch && Y < p.out_h && pc < p.px_w;
+        int8_t *dst = p.out + ((long long)n * p.out_rows_per_image + Y * p.out_grid_w + pc + p.out_row_off) *
+                                  p.out_pitch;
+        const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * c.acc_stride + 32 * wg);
+        int acc[16], b[16], d[16];
+        tmem_ld16(taddr, acc);
+        tmem_ld16(taddr + 16, b);
+        tmem_ld16(taddr + 32, d);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(c.acc_empty0 + 8 * a);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) acc[i] = max(max(acc[i], b[i]), d[i]);
+        float ks[16], bs[16];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const float4 kv = *reinterpret_cast<const float4 *>(&c.s_ks[4 * g]);
+            const float4 bv = *reinterpret_cast<const float4 *>(&c.s_bs[4 * g]);
+            ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+            bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+        }
+        uint32_t w[4];
+        requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+        if (valid) *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 }  // namespace
 
 // EXTRAS compiles in the residual add, the second output and the stored-code ReLU; layers that
@@ -698,7 +755,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // outputs may reuse buffers that the previous launch still reads
         asm volatile("griddepcontrol.wait;" ::: "memory");
         if constexpr (PXK) {  // multi-pixel rows: only built for the verified division
-            if (p.staged) {
+            if (p.hpool) {
+                if (p.relu_out) epilogue_hpool<true>(p, c, warp, lane);
+                else epilogue_hpool<false>(p, c, warp, lane);
+            } else if (p.staged) {
                 if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, true, KS>(p, c, warp, lane);
                 else epilogue_role<EXTRAS, kEpiFastDiv, false, true, true, KS>(p, c, warp, lane);
             } else {

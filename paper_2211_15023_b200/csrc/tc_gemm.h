@@ -46,6 +46,12 @@ struct TcGemmParams {
     // stored.  out_xmul scales X in the output row (px_per_row when out_pitch is one pixel).
     int px_per_row, px_cols, px_w;
     int out_xmul, out2_xmul;
+    // hpool = 1 (a conv whose only reader is a 3x3 stride-2 max-pool; 16 output channels; the GEMM
+    // row holds 9 output pixels, the last one the first of the next row): the epilogue takes the
+    // maximum of the ACCUMULATORS of pixels 2j, 2j+1, 2j+2 (j = 0..3) and requantises that -- the
+    // requantiser is non-decreasing in the accumulator, so max and requantisation commute -- and
+    // stores the 4 horizontally pooled pixels; px_w is then the pooled width, out_xmul = 4.
+    int hpool;
     int out_relu;     // clamp the stored codes at 0 (the only reader applies ReLU to its input)
     // optional second copy of the output in another layout: row = n * out2_rows_per_image +
     // Y * out2_grid_w + X + out2_row_off, `out2_pitch` bytes apart, ReLU'd if out2_relu

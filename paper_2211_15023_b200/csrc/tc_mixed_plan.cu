@@ -42,29 +42,27 @@ __global__ void maxpool_dual_kernel(const PoolDualParams q, long long total)
     int oy = (int)(t % q.OH);
     long long n = t / q.OH;
     uint32_t m[4] = {0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u};
-    const int8_t *win = q.in + ((n * q.in_hpitch + oy * q.stride + q.in_off_y) * q.in_wpitch + ox * q.stride +
+    const int8_t *win = q.in + ((n * q.in_hpitch + oy * q.stride + q.in_off_y) * q.in_wpitch + ox * q.stride_x +
                                 q.in_off_x) * q.C + g * 16;
     const int row_bytes = q.in_wpitch * q.C;
-    if (q.k == 3) {
+    auto take = [&](int ky, int kx) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(win + ky * row_bytes + kx * q.C));
+        m[0] = __vmaxs4(m[0], v.x);
+        m[1] = __vmaxs4(m[1], v.y);
+        m[2] = __vmaxs4(m[2], v.z);
+        m[3] = __vmaxs4(m[3], v.w);
+    };
+    if (q.k == 3 && q.kw == 3) {
 #pragma unroll
         for (int ky = 0; ky < 3; ++ky)
 #pragma unroll
-            for (int kx = 0; kx < 3; ++kx) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(win + ky * row_bytes + kx * q.C));
-                m[0] = __vmaxs4(m[0], v.x);
-                m[1] = __vmaxs4(m[1], v.y);
-                m[2] = __vmaxs4(m[2], v.z);
-                m[3] = __vmaxs4(m[3], v.w);
-            }
+            for (int kx = 0; kx < 3; ++kx) take(ky, kx);
+    } else if (q.k == 3 && q.kw == 1) {  // the producer has already pooled along x
+#pragma unroll
+        for (int ky = 0; ky < 3; ++ky) take(ky, 0);
     } else {
         for (int ky = 0; ky < q.k; ++ky)
-            for (int kx = 0; kx < q.k; ++kx) {
-                const uint4 v = __ldg(reinterpret_cast<const uint4 *>(win + ky * row_bytes + kx * q.C));
-                m[0] = __vmaxs4(m[0], v.x);
-                m[1] = __vmaxs4(m[1], v.y);
-                m[2] = __vmaxs4(m[2], v.z);
-                m[3] = __vmaxs4(m[3], v.w);
-            }
+            for (int kx = 0; kx < q.kw; ++kx) take(ky, kx);
     }
 #pragma unroll
     for (int o = 0; o < 2; ++o) {
@@ -317,12 +315,17 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
     // plain NHWC with rows of OW8 * 8 pixels
     const int W0 = p->in_w, H0 = p->in_h;
     const int PW = round_up(4 + W0 + 1, 8), PW8 = PW / 8, OW8 = (W0 + 7) / 8;
+    // Without the parity taps the first conv pools along x on its accumulators (TcGemmParams::hpool)
+    // and stores [n][H][OW8 * 4][C]: 4 pooled pixels per GEMM row.
+    const bool hpool_first = role[0] == TCFIRST && !keep && layers[0].out_c == 16 && layers[1].kh == 3 &&
+                             layers[1].kw == 3 && layers[1].stride == 2 && layers[1].pad == 0;
+    const int first_wpitch = hpool_first ? OW8 * 4 : OW8 * 8;
     int8_t *first_out = nullptr;
     if (role[0] == TCFIRST) {
         if ((st = alloc_zeroed(p, (size_t)p->max_batch * (H0 + 2) * PW * 4, &p->in_pad4)) != ACCERL_OK)
             return st;
         p->in_pad4_w = PW;
-        if ((st = alloc_zeroed(p, (size_t)p->max_batch * H0 * OW8 * 8 * layers[0].out_c, &first_out)) !=
+        if ((st = alloc_zeroed(p, (size_t)p->max_batch * H0 * first_wpitch * layers[0].out_c, &first_out)) !=
             ACCERL_OK)
             return st;
     }
@@ -389,7 +392,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             if (i == 1 && role[0] == TCFIRST) {
                 q.in = first_out;
                 q.in_hpitch = L.in_h;
-                q.in_wpitch = OW8 * 8;
+                q.in_wpitch = first_wpitch;
             } else if (fin.slot) {
                 q.in = fin.p_slot;
                 q.in_hpitch = L.in_h + 2;
@@ -414,6 +417,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             else if (fout.slot_relu) return bail();
             q.H = L.in_h; q.W = L.in_w; q.C = L.in_c; q.OH = L.out_h; q.OW = L.out_w;
             q.k = d.kh; q.stride = d.stride;
+            q.kw = hpool_first && i == 1 ? 1 : d.kw;
+            q.stride_x = hpool_first && i == 1 ? 1 : d.stride;
             p->pools.push_back(q);
             s.kind = Step::POOL_DUAL;
             s.tc = (int)p->pools.size() - 1;
@@ -434,7 +439,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         TcGemmParams &g = ts.prm;
         const bool logits = (d.flags & ACCERL_LOGITS) != 0;
         const int P = role[i] == TCPX ? tcpx_pixels(d) : 0;  // output pixels per GEMM row
-        const int n_total = role[i] == TCFIRST ? 8 * d.out_c : (P ? P * d.out_c : round_up(d.out_c, 16));
+        const int first_px = hpool_first ? 9 : 8;  // output pixels per GEMM row of the first conv
+        const int n_total = role[i] == TCFIRST ? first_px * d.out_c : (P ? P * d.out_c : round_up(d.out_c, 16));
         g.sub = 1;
         g.max_sub = 1;
         g.out_xmul = g.out2_xmul = 1;
@@ -469,7 +475,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                     const int j = ky * 2 + d8;
                     g.row_off[j] = ky * PW8 + d8;
                     g.col_off[j] = 0;
-                    for (int px = 0; px < 8; ++px)
+                    for (int px = 0; px < first_px; ++px)
                         for (int oc = 0; oc < d.out_c; ++oc)
                             for (int pin = 0; pin < 8; ++pin) {
                                 const int kx = d8 * 8 + pin - px - 3;
@@ -482,9 +488,9 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             a_ptr = p->in_pad4;
             a_rows_total = (long long)p->max_batch * (H0 + 2) * PW8;
             row_bytes = 32;
-            // per-column scales: the channel's, repeated for the 8 pixels
+            // per-column scales: the channel's, repeated for the pixels of the row
             std::vector<float> ks(n_total), bs(n_total);
-            for (int px = 0; px < 8; ++px)
+            for (int px = 0; px < first_px; ++px)
                 for (int oc = 0; oc < d.out_c; ++oc) {
                     volatile float k = d.s_in * d.s_w[oc];
                     ks[px * d.out_c + oc] = k;
@@ -607,12 +613,16 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         } outs[4];
         int n_out = 0;
         if (role[i] == TCFIRST) {
-            outs[n_out++] = OutSpec{first_out, L.out_h * OW8, OW8, 0, n_total, 0, 1};
-            TapDesc &td = p->taps[i + 1];
-            td.ptr = first_out;
-            td.pitch = d.out_c;
-            td.hpitch = L.out_h;
-            td.wpitch = OW8 * 8;
+            if (hpool_first) {  // in pooled pixels; no tap (the un-pooled tensor is never stored)
+                outs[n_out++] = OutSpec{first_out, L.out_h * first_wpitch, first_wpitch, 0, d.out_c, 0, 4};
+            } else {
+                outs[n_out++] = OutSpec{first_out, L.out_h * OW8, OW8, 0, n_total, 0, 1};
+                TapDesc &td = p->taps[i + 1];
+                td.ptr = first_out;
+                td.pitch = d.out_c;
+                td.hpitch = L.out_h;
+                td.wpitch = OW8 * 8;
+            }
         } else if (!logits) {
             // Row pitch = one pixel of the stored form; a multi-pixel GEMM row starts at pixel
             // X * P and its columns run on over the following pixels.
@@ -687,8 +697,15 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             if (st != ACCERL_OK) return st;
             g.fast_div = ok ? 1 : 0;
         }
-        g.split_cols = g.n_tile > 128 ? 1 : 0;
+        g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first)) ? 1 : 0;
         if (role[i] == TCPX && !g.fast_div) return bail();  // multi-pixel rows need the verified division
+        if (role[i] == TCFIRST && hpool_first) {
+            if (!g.fast_div) return bail();
+            g.hpool = 1;
+            g.px_per_row = 8;  // selects the multi-pixel kernel
+            g.px_cols = d.out_c;
+            g.px_w = (W0 - 3) / 2 + 1;  // pooled width
+        }
         // layers that also read a residual or write a second form: collect the rows in shared memory
         // and move whole 128-byte lines (the load/store path bounds them otherwise)
         g.staged = (role[i] == TCPX && g.n_tile == 128 && (g.skip || g.out2)) ? 1 : 0;
