@@ -439,15 +439,18 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
             r -= p.rows_per_image;
         }
         const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
-        const int pc = X * 4 + wg;  // pooled column
+        // warpgroup -> (pooled pixel of the row, 16-channel piece): 4 x 1 at 16 channels, 2 x 2 at 32
+        const int hpc = p.px_cols >> 4, ox = wg / hpc, half = wg - ox * hpc;
+        const int pc = X * (4 / hpc) + ox;  // pooled column
         const bool valid = n < p.batch && Y < p.out_h && pc < p.px_w;
         int8_t *dst = p.out + ((long long)n * p.out_rows_per_image + Y * p.out_grid_w + pc + p.out_row_off) *
-                                  p.out_pitch;
-        const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * c.acc_stride + 32 * wg);
+                                  p.out_pitch + 16 * half;
+        const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) +
+                               (uint32_t)(a * c.acc_stride + 2 * ox * p.px_cols + 16 * half);
         int acc[16], b[16], d[16];
         tmem_ld16(taddr, acc);
-        tmem_ld16(taddr + 16, b);
-        tmem_ld16(taddr + 32, d);
+        tmem_ld16(taddr + p.px_cols, b);
+        tmem_ld16(taddr + 2 * p.px_cols, d);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
@@ -457,8 +460,8 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
         float ks[16], bs[16];
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
-            const float4 kv = *reinterpret_cast<const float4 *>(&c.s_ks[4 * g]);
-            const float4 bv = *reinterpret_cast<const float4 *>(&c.s_bs[4 * g]);
+            const float4 kv = *reinterpret_cast<const float4 *>(&c.s_ks[16 * half + 4 * g]);
+            const float4 bv = *reinterpret_cast<const float4 *>(&c.s_bs[16 * half + 4 * g]);
             ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
             bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
         }

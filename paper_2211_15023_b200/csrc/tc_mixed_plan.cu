@@ -160,12 +160,13 @@ enum Role { GENERIC, POOL, TCCONV, TCPX, TCFC, TCFIRST };
 
 struct Forms {  // which stored forms of a tensor its readers need
     bool plain = false, plain_relu = false, pad = false, pad_relu = false, slot = false, slot_relu = false;
+    bool hp = false;  // pooled along x by its producer: [n][H][hp_w][C], read by a max-pool only
     int8_t *p_plain = nullptr, *p_plain_relu = nullptr, *p_pad = nullptr, *p_slot = nullptr,
-           *p_slot_relu = nullptr;
+           *p_slot_relu = nullptr, *p_hp = nullptr;
     int count() const
     {
         return (plain ? 1 : 0) + (plain_relu ? 1 : 0) + ((pad || pad_relu) ? 1 : 0) + (slot ? 1 : 0) +
-               (slot_relu ? 1 : 0);
+               (slot_relu ? 1 : 0) + (hp ? 1 : 0);
     }
 };
 
@@ -188,6 +189,9 @@ bool tcconv_ok(const accerl_layer_desc &d)
            (d.in_c == 16 || d.in_c == 32) && d.out_c % 16 == 0 && d.out_c <= 256 &&
            128 + 2 * (d.in_w + 2) + 2 <= 256;
 }
+
+// stored pixels per row of a tensor that its producer (P pixels per GEMM row) has pooled along x
+int hp_width(int W, int P) { return slot_pw(W) / P * (P / 2); }
 
 accerl_status alloc_zeroed(accerl_policy *p, size_t bytes, int8_t **out)
 {
@@ -266,7 +270,20 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         } else if (role[j] == POOL) {
             if (relu_in) return ACCERL_OK;
             // a pool reads whatever its producer writes naturally
-            (role[j - 1] == TCPX ? f.slot : f.plain) = true;
+            // a pool reads whatever its producer writes naturally; a multi-pixel conv that only feeds
+            // a 3x3 stride-2 pool pools along x itself (TcGemmParams::hpool)
+            bool only_reader = !keep && j >= 1 && role[j - 1] == TCPX && d.kh == 3 && d.kw == 3 &&
+                               d.stride == 2 && d.pad == 0 && layers[j - 1].skip_from < 0;
+            for (int q = 0; q < n_layers && only_reader; ++q)
+                if (layers[q].skip_from == j - 1) only_reader = false;
+            if (only_reader) {
+                const int P = tcpx_pixels(layers[j - 1]);
+                // (measured: worth it while the wider K window still fits four 32-byte steps per tap row)
+                only_reader = (P / 2) * (layers[j - 1].out_c / 16) == 4 && (P + 1) * layers[j - 1].out_c <= 256 &&
+                              (P + 3) * layers[j - 1].in_c <= 128;
+            }
+            if (only_reader) f.hp = true;
+            else (role[j - 1] == TCPX ? f.slot : f.plain) = true;
         } else if (role[j] == TCCONV) {
             (relu_in ? f.pad_relu : f.pad) = true;
         } else if (role[j] == TCPX) {
@@ -306,6 +323,9 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             (st = alloc_zeroed(p, (size_t)p->max_batch * (H + 2) * (W + 2) * 32, &f.p_pad)) != ACCERL_OK)
             return st;
         const size_t slot_bytes = (size_t)p->max_batch * (H + 2) * slot_pw(W) * C;
+        if (f.hp && (st = alloc_zeroed(p, (size_t)p->max_batch * H * hp_width(W, tcpx_pixels(layers[t - 1])) * C,
+                                       &f.p_hp)) != ACCERL_OK)
+            return st;
         if (f.slot && (st = alloc_zeroed(p, slot_bytes, &f.p_slot)) != ACCERL_OK) return st;
         if (f.slot_relu && (st = alloc_zeroed(p, slot_bytes, &f.p_slot_relu)) != ACCERL_OK) return st;
     }
@@ -393,6 +413,10 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                 q.in = first_out;
                 q.in_hpitch = L.in_h;
                 q.in_wpitch = first_wpitch;
+            } else if (fin.hp) {
+                q.in = fin.p_hp;
+                q.in_hpitch = L.in_h;
+                q.in_wpitch = hp_width(L.in_w, tcpx_pixels(layers[i - 1]));
             } else if (fin.slot) {
                 q.in = fin.p_slot;
                 q.in_hpitch = L.in_h + 2;
@@ -417,8 +441,9 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             else if (fout.slot_relu) return bail();
             q.H = L.in_h; q.W = L.in_w; q.C = L.in_c; q.OH = L.out_h; q.OW = L.out_w;
             q.k = d.kh; q.stride = d.stride;
-            q.kw = hpool_first && i == 1 ? 1 : d.kw;
-            q.stride_x = hpool_first && i == 1 ? 1 : d.stride;
+            const bool pre_pooled = (hpool_first && i == 1) || fin.hp;
+            q.kw = pre_pooled ? 1 : d.kw;
+            q.stride_x = pre_pooled ? 1 : d.stride;
             p->pools.push_back(q);
             s.kind = Step::POOL_DUAL;
             s.tc = (int)p->pools.size() - 1;
@@ -438,9 +463,11 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         memset(&ts.prm, 0, sizeof(ts.prm));
         TcGemmParams &g = ts.prm;
         const bool logits = (d.flags & ACCERL_LOGITS) != 0;
-        const int P = role[i] == TCPX ? tcpx_pixels(d) : 0;  // output pixels per GEMM row
+        const int P = role[i] == TCPX ? tcpx_pixels(d) : 0;  // stored pixels per GEMM row
+        const bool hp_out = role[i] == TCPX && fout.hp;       // pools along x: one output pixel more per row
+        const int Pout = hp_out ? P + 1 : P;
         const int first_px = hpool_first ? 9 : 8;  // output pixels per GEMM row of the first conv
-        const int n_total = role[i] == TCFIRST ? first_px * d.out_c : (P ? P * d.out_c : round_up(d.out_c, 16));
+        const int n_total = role[i] == TCFIRST ? first_px * d.out_c : (P ? Pout * d.out_c : round_up(d.out_c, 16));
         g.sub = 1;
         g.max_sub = 1;
         g.out_xmul = g.out2_xmul = 1;
@@ -505,7 +532,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             // GEMM row = P stored pixels; its K window is those and the next two pixels, for each
             // of the three rows ky: steps of 32 bytes, the last one or two from the GEMM row after.
             const int PW = slot_pw(d.in_w), G = PW / P, row = P * d.in_c;
-            const int first_ks = row / 32, n_ks = (P + 2) * d.in_c / 32;
+            const int first_ks = row / 32, n_ks = ((Pout + 2) * d.in_c + 31) / 32;
             g.chunk_bytes = row;
             g.kstep_list = 1;
             g.n_chunks = 3 * n_ks;
@@ -522,7 +549,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                     const int j = ky * n_ks + ks;
                     g.row_off[j] = ky * G + (ks < first_ks ? 0 : 1);
                     g.col_off[j] = 32 * (ks < first_ks ? ks : ks - first_ks);
-                    for (int px = 0; px < P; ++px)
+                    for (int px = 0; px < Pout; ++px)
                         for (int oc = 0; oc < d.out_c; ++oc)
                             for (int kk = 0; kk < 32; ++kk) {
                                 const int wb = 32 * ks + kk, pin = wb / d.in_c, c = wb % d.in_c;
@@ -539,7 +566,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             // per-column scales and residual multipliers: the channel's, repeated for the P pixels
             std::vector<float> ks(n_total), bs(n_total);
             std::vector<int32_t> sm(n_total, 0);
-            for (int px = 0; px < P; ++px)
+            for (int px = 0; px < Pout; ++px)
                 for (int oc = 0; oc < d.out_c; ++oc) {
                     volatile float k = d.s_in * d.s_w[oc];
                     ks[px * d.out_c + oc] = k;
@@ -634,6 +661,10 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                 if (P && d.out_c != 32) return bail();
                 outs[n_out++] = OutSpec{fout.p_pad, (H + 2) * (W + 2), W + 2, W + 3, 32, fout.pad_relu ? 1 : 0, xm};
             }
+            if (fout.hp) {
+                const int hw = hp_width(W, P);
+                outs[n_out++] = OutSpec{fout.p_hp, H * hw, hw, 0, L.out_cp, 0, P / 2};
+            }
             if (fout.slot) outs[n_out++] = OutSpec{fout.p_slot, (H + 2) * SW, SW, SW + 1, L.out_cp, 0, xm};
             if (fout.slot_relu)
                 outs[n_out++] = OutSpec{fout.p_slot_relu, (H + 2) * SW, SW, SW + 1, L.out_cp, 1, xm};
@@ -697,8 +728,12 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             if (st != ACCERL_OK) return st;
             g.fast_div = ok ? 1 : 0;
         }
-        g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first)) ? 1 : 0;
+        g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first) || hp_out) ? 1 : 0;
         if (role[i] == TCPX && !g.fast_div) return bail();  // multi-pixel rows need the verified division
+        if (hp_out) {
+            g.hpool = 1;
+            g.px_w = (L.out_w - 3) / 2 + 1;  // pooled width
+        }
         if (role[i] == TCFIRST && hpool_first) {
             if (!g.fast_div) return bail();
             g.hpool = 1;
@@ -714,7 +749,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         g.status = p->status_word;
         g.trace_slot = (int)p->tc_steps.size() % 8;
         const int b_bytes = g.kstep_list ? 32 : g.chunk_bytes;  // bytes of a weight row per chunk
-        ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * b_bytes <= 96 * 1024;
+        ts.resident_b = g.n_tiles == 1 && (size_t)g.n_chunks * n_total * b_bytes <= 112 * 1024;
         if (g.shifted && !ts.resident_b) return bail();
         if (!tc_choose_pipeline(g, ts.resident_b)) {
             if (g.shifted) return bail();
