@@ -199,6 +199,31 @@ def test_multi_pixel_rows_ragged_widths(hw):
         g.close()
 
 
+def test_tensor_core_logits_layer_with_many_actions():
+    """More than 32 actions: the last layer cannot run fused with the sampler, so the tensor-core
+    kernel writes the fp32 logits itself and the wide sampler follows."""
+    import paper_2211_15023_b200 as P
+    rng = np.random.default_rng(31)
+    layers = W.nature_cnn(16, 32, 32, 256, actions=40)
+    params = [dict(w=(rng.standard_normal((l["out_c"], l["in_c"], l["kh"], l["kw"])) *
+                      np.sqrt(2.0 / (l["in_c"] * l["kh"] * l["kw"]))).astype(np.float32),
+                   bias=rng.standard_normal(l["out_c"]).astype(np.float32) * 0.05) for l in layers]
+    calib = rng.integers(0, 256, (64, 4, 84, 84), dtype=np.uint8)
+    pol = oracle.calibrate("u8", (4, 84, 84), layers, params, calib)
+    b = 45
+    obs = rng.integers(0, 256, (b, 4, 84, 84), dtype=np.uint8)
+    u = rng.random(b, dtype=np.float32)
+    ref = oracle.forward(pol, obs, u)
+    for flags in (1, 0):
+        g = P.Policy(pol, b, flags=flags)
+        plan = g.info()["plan"]
+        assert "tc_gemm_kernel" in plan and "sample_wide_kernel" in plan
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        g.check()
+        compare(ref, *out, taps=g.read_activation if flags else None)
+        g.close()
+
+
 def test_exact_ties_on_the_tensor_core_path():
     """Power-of-two scales make many epilogue quotients land exactly on k + 0.5: the requantiser
     must round them to even exactly as the IEEE divide + rintf of the definition does."""
