@@ -10,12 +10,19 @@
 // would leave the image are computed and thrown away by the epilogue.
 //
 // Roles inside a CTA (768 threads): warps 0..3 issue TMA loads, warps 4..7 issue the MMAs (warp 4
-// owns the tensor-memory allocation), warps 8..23 are four epilogue warpgroups that drain accumulators (each warp its own
-// 32-lane quarter of tensor memory), requantise and store; the warpgroups take tiles in turn,
-// or for wide tiles a quarter of the columns each.  The epilogue is latency bound per warp, so
-// four warps per scheduler are what keeps the issue slots busy.  The kernel is persistent: CTAs stride over the tile list, smem stages
-// and accumulator stages are ring buffers guarded by mbarriers.  Every wait is bounded; a wait
-// that gives up sets the policy's status word and all roles leave.
+// owns the tensor-memory allocation), warps 8..23 are four epilogue warpgroups that drain
+// accumulators (each warp its own 32-lane quarter of tensor memory), requantise and store; the
+// warpgroups take tiles in turn, or for wide tiles a quarter of the columns each.  The epilogue is
+// latency bound per warp, so four warps per scheduler are what keeps the issue slots busy.  The
+// kernel is persistent: CTAs stride over the tile list, smem stages and accumulator stages are ring
+// buffers guarded by mbarriers.  Every wait is bounded; a wait that gives up sets the policy's
+// status word and all roles leave.
+//
+// Variants, all chosen per launch from TcGemmParams: several output pixels per GEMM row with
+// banded weights and a list of 32-byte K steps (kstep_list, px_per_row), rows collected in shared
+// memory and stored as whole lines (staged), max-pooling along x on the accumulators (hpool),
+// the K loop of a tile split over the issuing warps (ksplit).  The launch is a programmatic
+// dependent launch: set-up overlaps the previous launch's tail.
 #include <cuda.h>
 
 #include "epilogue.cuh"

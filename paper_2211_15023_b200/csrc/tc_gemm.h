@@ -69,7 +69,7 @@ struct TcGemmParams {
     float s_out, inv_s_out;
     int fast_div;  // 1: the three-step division has been verified for this s_out (epilogue.cuh)
     int relu_out;
-    int split_cols;  // 1: both epilogue warpgroups share a tile (half the columns each)
+    int split_cols;  // 1: the four epilogue warpgroups share a tile (a quarter of the columns each)
     // 1: rows leave through a shared-memory tile per warp, eight lanes per row (needs n_tile = 128,
     // rows of 128 contiguous output bytes, the verified three-step division, no split_cols)
     int staged;
