@@ -418,16 +418,21 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
     }
 }
 
-// Epilogue for hpool layers (see TcGemmParams::hpool): all four warpgroups share every tile,
-// warpgroup j produces pooled pixel j of each row from the accumulators of pixels 2j .. 2j+2.
+// Epilogue for hpool layers (see TcGemmParams::hpool): the warpgroups work in two pairs, each pair
+// on every other tile (two tiles are drained at a time, one per accumulator stage); inside a pair a
+// warp produces two of the row's four (pooled pixel, 16-channel piece) items, each from the
+// accumulators of pixels 2j .. 2j+2.
 template <bool RELU>
 __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
 {
     const int q = warp & 3, wg = (warp - kProdWarps - kMmaWarps) >> 2;
+    const int pair = wg >> 1, side = wg & 1;
     const float s_out = p.s_out, inv_s_out = p.inv_s_out;
+    const int hpc = p.px_cols >> 4;  // 16-channel pieces per pixel: 1 or 2
     int tile_i = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < c.total_tiles && ok; t += gridDim.x, ++tile_i) {
+        if ((tile_i & 1) != pair) continue;
         const int a = tile_i & (c.n_acc - 1);
         const uint32_t apar = (tile_i >> p.n_acc_log2) & 1;
         ok = mbar_wait(c.acc_full0 + 8 * a, apar, c.abort_flag, p.status, 16);
@@ -446,35 +451,40 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
             r -= p.rows_per_image;
         }
         const int Y = (int)__umulhi((unsigned)r, p.grid_w_magic), X = r - Y * p.grid_w;
-        // warpgroup -> (pooled pixel of the row, 16-channel piece): 4 x 1 at 16 channels, 2 x 2 at 32
-        const int hpc = p.px_cols >> 4, ox = wg / hpc, half = wg - ox * hpc;
-        const int pc = X * (4 / hpc) + ox;  // pooled column
-        const bool valid = n < p.batch && Y < p.out_h && pc < p.px_w;
-        int8_t *dst = p.out + ((long long)n * p.out_rows_per_image + Y * p.out_grid_w + pc + p.out_row_off) *
-                                  p.out_pitch + 16 * half;
-        const uint32_t taddr = c.tmem_base + ((uint32_t)(q * 32) << 16) +
-                               (uint32_t)(a * c.acc_stride + 2 * ox * p.px_cols + 16 * half);
-        int acc[16], b[16], d[16];
-        tmem_ld16(taddr, acc);
-        tmem_ld16(taddr + p.px_cols, b);
-        tmem_ld16(taddr + 2 * p.px_cols, d);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) mbar_arrive(c.acc_empty0 + 8 * a);
+        const bool row_ok = n < p.batch && Y < p.out_h;
+        int8_t *dst_row = p.out + ((long long)n * p.out_rows_per_image + Y * p.out_grid_w + X * (4 / hpc) +
+                                   p.out_row_off) * p.out_pitch;
+        const uint32_t tbase = c.tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * c.acc_stride);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) acc[i] = max(max(acc[i], b[i]), d[i]);
-        float ks[16], bs[16];
+        for (int item = 0; item < 2; ++item) {
+            // 16 channels per pixel: pooled pixels 2 * side + item; 32: pixel `side`, piece `item`
+            const int ox = hpc == 1 ? 2 * side + item : side, half = hpc == 1 ? 0 : item;
+            const uint32_t taddr = tbase + (uint32_t)(2 * ox * p.px_cols + 16 * half);
+            int acc[16], b[16], d[16];
+            tmem_ld16(taddr, acc);
+            tmem_ld16(taddr + p.px_cols, b);
+            tmem_ld16(taddr + 2 * p.px_cols, d);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (item == 1) {  // the last read of the stage: hand it back
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(c.acc_empty0 + 8 * a);
+            }
 #pragma unroll
-        for (int g = 0; g < 4; ++g) {
-            const float4 kv = *reinterpret_cast<const float4 *>(&c.s_ks[16 * half + 4 * g]);
-            const float4 bv = *reinterpret_cast<const float4 *>(&c.s_bs[16 * half + 4 * g]);
-            ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
-            bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+            for (int i = 0; i < 16; ++i) acc[i] = max(max(acc[i], b[i]), d[i]);
+            float ks[16], bs[16];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                const float4 kv = *reinterpret_cast<const float4 *>(&c.s_ks[16 * half + 4 * g]);
+                const float4 bv = *reinterpret_cast<const float4 *>(&c.s_bs[16 * half + 4 * g]);
+                ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
+            }
+            uint32_t w[4];
+            requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+            if (row_ok && X * (4 / hpc) + ox < p.px_w)
+                *reinterpret_cast<uint4 *>(dst_row + ox * p.out_pitch + 16 * half) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        uint32_t w[4];
-        requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
-        if (valid) *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -548,7 +558,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < n_acc; ++a) {
             mbar_init(smem_u32(&bars.acc_full[a]), (!RESIDENT_B && p.ksplit) ? p.n_mma : 1);
-            mbar_init(smem_u32(&bars.acc_empty[a]), p.split_cols ? 4 * kEpiGroups : 4);
+            mbar_init(smem_u32(&bars.acc_empty[a]), p.hpool ? 8 : (p.split_cols ? 4 * kEpiGroups : 4));
         }
         mbar_init(smem_u32(&bars.b_ready), 1);
         bars.abort_flag = 0;
