@@ -290,6 +290,13 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             prm.batch = B;
             prm.m_tiles = (int)(((long long)B * prm.rows_per_image + 127) / 128);
             prm.logits = prm.logits_mode ? logits_dev : nullptr;
+            if (prm.fuse_ingest) {
+                if ((uintptr_t)obs_dev & 15) {
+                    set_error("act: this plan reads the frames with 16-byte bulk copies; obs_dev must be 16-byte aligned");
+                    return ACCERL_ERR_INVALID_ARG;
+                }
+                prm.obs = (const uint8_t *)obs_dev;
+            }
             ACCERL_CUDA_TRY(tc_launch(t.map_a, t.map_b, prm, t.resident_b, p->sm_count, st));
             break;
         }
@@ -530,6 +537,9 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         }
         if ((st = upload(p, lut, &p->lut)) != ACCERL_OK) return fail(st);
         p->ingest_arith = fit_ingest_line(lut.data(), &p->ingest_mul, &p->ingest_add) ? 1 : 0;
+        p->ingest_shift1 = true;
+        for (int u = 0; u < 256; ++u)
+            if (lut[u] != (u >> 1)) p->ingest_shift1 = false;
         // the float form of the line (measured faster in the NHWC kernel, slower in the space-to-depth one)
         p->ingest_float = p->ingest_arith == 1 &&
                           fit_ingest_float_line(lut.data(), p->ingest_mul, p->ingest_add, &p->ingest_fa,

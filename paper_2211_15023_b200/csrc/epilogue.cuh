@@ -136,6 +136,37 @@ __device__ __forceinline__ void requant16_fastdiv(const int (&acc)[16], const fl
 }
 
 // Four frame bytes (byte `dx` of the words p0..p3, one per channel plane) -> four int8 codes in one
+// word, channel 0 in the low byte, by the fixed-point line q = min((u * mul + add) >> 24, 127).
+template <bool CLAMP>
+__device__ __forceinline__ uint32_t ingest_fixed_line4(uint32_t p0, uint32_t p1, uint32_t p2, uint32_t p3,
+                                                       int dx, uint32_t mul, uint32_t add)
+{
+    const uint32_t sel = 0x4440u + (uint32_t)dx;  // byte dx, zero extended
+    const uint32_t r0 = __byte_perm(p0, 0, sel) * mul + add, r1 = __byte_perm(p1, 0, sel) * mul + add;
+    const uint32_t r2 = __byte_perm(p2, 0, sel) * mul + add, r3 = __byte_perm(p3, 0, sel) * mul + add;
+    // top bytes of the four multiply-adds
+    const uint32_t lo = __byte_perm(r0, r1, 0x0073), hi = __byte_perm(r2, r3, 0x0073);
+    const uint32_t codes = __byte_perm(lo, hi, 0x5410);
+    return CLAMP ? __vminu4(codes, 0x7f7f7f7fu) : codes;  // without: the host saw the line stay <= 127
+}
+
+// The table q(u) = u >> 1 (what the input quantiser is when s_input = 1/127, the scale max-abs
+// calibration gives whenever a calibration frame contains a 255): four words of four bytes each
+// (one per channel plane, bytes = 4 pixels) -> four words of (channel 0..3) codes per pixel.
+// Halving is done on all four bytes of a word at once; the rest is a 4 x 4 byte transpose.
+__device__ __forceinline__ uint4 ingest_shift_line16(uint32_t p0, uint32_t p1, uint32_t p2, uint32_t p3)
+{
+    p0 = (p0 >> 1) & 0x7f7f7f7fu;
+    p1 = (p1 >> 1) & 0x7f7f7f7fu;
+    p2 = (p2 >> 1) & 0x7f7f7f7fu;
+    p3 = (p3 >> 1) & 0x7f7f7f7fu;
+    const uint32_t a = __byte_perm(p0, p1, 0x5140), b = __byte_perm(p0, p1, 0x7362);  // c0 c1 of pixels 0,1 / 2,3
+    const uint32_t c = __byte_perm(p2, p3, 0x5140), d = __byte_perm(p2, p3, 0x7362);  // c2 c3
+    return make_uint4(__byte_perm(a, c, 0x5410), __byte_perm(a, c, 0x7632), __byte_perm(b, d, 0x5410),
+                      __byte_perm(b, d, 0x7632));
+}
+
+// Four frame bytes (byte `dx` of the words p0..p3, one per channel plane) -> four int8 codes in one
 // word, channel 0 in the low byte, without integer multiplies: a byte permute builds the float
 // 128 + u/256 from byte u, two packed float operations map it onto 1.5 * 2^23 + code (rounded to
 // nearest by the addition itself), and the codes are the low bytes of the bit patterns.  The two

@@ -130,6 +130,7 @@ struct accerl_policy {
     int8_t *lut = nullptr;                // device, 256-entry uint8 -> int8 input table
     int ingest_arith = 0;                 // the table is the line min((u * mul + add) >> 24, 127)
     uint32_t ingest_mul = 0, ingest_add = 0;
+    bool ingest_shift1 = false;           // the table is exactly u >> 1 (s_input = 1/127)
     bool ingest_float = false;            // the same line in float form: code = low byte of fma(f - c1, A, 1.5 * 2^23)
     uint32_t ingest_fa = 0, ingest_fc1 = 0;  // bit patterns of A and c1
     int *status_word = nullptr;           // device, set by kernels whose bounded waits give up

@@ -118,6 +118,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// untiled bulk copy global -> shared (16-byte aligned addresses, size a multiple of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
 // shared-memory matrix descriptor, K-major, swizzled rows of `chunk_bytes` (32 / 64 / 128)
 __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr, int chunk_bytes)
 {
@@ -189,6 +198,8 @@ struct __align__(8) Barriers {
     uint64_t full[kTcMaxStages], empty[kTcMaxStages];
     uint64_t acc_full[kTcMaxAccStages], acc_empty[kTcMaxAccStages];
     uint64_t b_ready;
+    uint64_t raw_full[kProdWarps];   // fused ingest: the raw frame strips of a step have landed
+    uint64_t conv_done[kProdWarps];  // fused ingest: the issuing warp has built its tile
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -488,13 +499,57 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
     }
 }
 
+// Fused input stage: one operand tile (a_rows rows from GEMM row g0 on) from the raw frame strips
+// in shared memory, one lane per row: sixteen 4-byte loads (4 image rows x 4 channel planes), 64
+// quantised bytes in (dy, dx, c) order, stored as four 16-byte pieces under the 64-byte swizzle
+// (piece index XOR address bits 7..8).  Rows past the last state are zero.  t0 = position of g0
+// relative to the first column of the first grid row held in `raw`.
+template <int MODE>  // 0: line without the min, 1: line with it, 2: q = u >> 1
+__device__ __forceinline__ void convert_tile(const TcGemmParams &p, const uint8_t *raw, uint8_t *tile,
+                                             long long g0, int t0, long long total_rows, int lane)
+{
+    const int Ws = p.grid_w, strip = 4 * p.in_w;
+    for (int rr = lane; rr < p.a_rows; rr += 32) {
+        const unsigned tt = (unsigned)(t0 + rr);
+        const int Rrel = (int)__umulhi(tt, p.grid_w_magic), X = (int)tt - Rrel * Ws;
+        uint4 q[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
+                      make_uint4(0, 0, 0, 0)};
+        if (g0 + rr < total_rows) {
+            uint32_t w[4][4];  // [dy][channel]
+#pragma unroll
+            for (int dy = 0; dy < 4; ++dy)
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    w[dy][c] = *reinterpret_cast<const uint32_t *>(raw + (c * p.raw_rows + Rrel) * strip +
+                                                                  dy * p.in_w + 4 * X);
+#pragma unroll
+            for (int dy = 0; dy < 4; ++dy) {
+                if (MODE == 2) {
+                    q[dy] = ingest_shift_line16(w[dy][0], w[dy][1], w[dy][2], w[dy][3]);
+                } else {
+                    constexpr bool CL = MODE == 1;
+                    q[dy] = make_uint4(
+                        ingest_fixed_line4<CL>(w[dy][0], w[dy][1], w[dy][2], w[dy][3], 0, p.ingest_mul, p.ingest_add),
+                        ingest_fixed_line4<CL>(w[dy][0], w[dy][1], w[dy][2], w[dy][3], 1, p.ingest_mul, p.ingest_add),
+                        ingest_fixed_line4<CL>(w[dy][0], w[dy][1], w[dy][2], w[dy][3], 2, p.ingest_mul, p.ingest_add),
+                        ingest_fixed_line4<CL>(w[dy][0], w[dy][1], w[dy][2], w[dy][3], 3, p.ingest_mul, p.ingest_add));
+                }
+            }
+        }
+#pragma unroll
+        for (int dy = 0; dy < 4; ++dy)
+            *reinterpret_cast<uint4 *>(tile + rr * 64 + ((dy ^ ((rr >> 1) & 3)) << 4)) = q[dy];
+    }
+}
+
 }  // namespace
 
 // EXTRAS compiles in the residual add, the second output and the stored-code ReLU; layers that
 // use none of them run the leaner instantiation (the epilogue is bound by instruction issue).
+// FUSE is the first conv with the input stage inside (TcGemmParams::fuse_ingest).
 // PXK is the kernel for rows of several output pixels; it is kept apart so that its epilogue
 // variants do not weigh on the register allocation of the others.
-template <bool RESIDENT_B, bool EXTRAS, bool PXK>
+template <bool RESIDENT_B, bool EXTRAS, bool PXK, bool FUSE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcGemmParams p)
@@ -561,6 +616,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             mbar_init(smem_u32(&bars.acc_empty[a]), p.hpool ? 8 : (p.split_cols ? 4 * kEpiGroups : 4));
         }
         mbar_init(smem_u32(&bars.b_ready), 1);
+        for (int i = 0; i < kProdWarps; ++i) {
+            mbar_init(smem_u32(&bars.raw_full[i]), 1);
+            mbar_init(smem_u32(&bars.conv_done[i]), 1);
+        }
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -621,11 +680,78 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int base_slot = 0;  // ring position of the current tile inside this warp's ring
         uint32_t base_phase = 0;
         int t = blockIdx.x + pw * gridDim.x;
+        if constexpr (FUSE) {
+            // Fused input stage.  A step's rows are space-to-depth(4) positions (R, X) of uint8 NCHW
+            // frames, R = image * grid_h + Y.  The four image rows 4Y .. 4Y+3 of one channel are
+            // in_w * 4 contiguous, 16-byte aligned bytes and consecutive Y of an image follow each
+            // other, so the raw bytes under a step arrive with at most two bulk copies per channel
+            // plane.  This warp then builds the step's first operand tile, the ring's issuing warp
+            // the second (or the upper half of a single one); both fence their writes to the async
+            // proxy.  The ring has one stage and one raw buffer: the next step's strips are fetched
+            // as soon as both warps have read the current ones, while the MMAs of this step run.
+            const int Ws = p.grid_w, Hs = p.rows_per_image / Ws, strip = 4 * p.in_w;
+            const long long total_rows = (long long)p.batch * p.rows_per_image;
+            const int raw_bytes = (4 * p.raw_rows * strip + 127) & ~127;
+            uint8_t *raw = stages + (size_t)n_stages * stage_bytes + (size_t)pw * raw_bytes;
+            const uint32_t raw_bar = smem_u32(&bars.raw_full[pw]);
+            const int step_rows = (SUB - 1) * kTileM + p.a_rows;
+            auto fetch = [&](int step) {  // elected lane: the raw strips under `step`
+                const long long g0 = (long long)step * kTileM * SUB;
+                long long g1 = g0 + step_rows;
+                if (g1 > total_rows) g1 = total_rows;
+                if (g1 <= g0) {
+                    mbar_expect_tx(raw_bar, 0);
+                    return;
+                }
+                const int R0 = (int)(g0 / Ws), R1 = (int)((g1 - 1) / Ws);
+                mbar_expect_tx(raw_bar, (uint32_t)(4 * (R1 - R0 + 1) * strip));
+                const uint32_t dst0 = smem_u32(raw);
+                int R = R0;
+                while (R <= R1) {  // runs of grid rows inside one image
+                    const int n = R / Hs;
+                    int Re = (n + 1) * Hs - 1;
+                    if (Re > R1) Re = R1;
+                    const int Y = R - n * Hs, cnt = Re - R + 1;
+                    for (int c = 0; c < 4; ++c)
+                        bulk_load(dst0 + (uint32_t)((c * p.raw_rows + (R - R0)) * strip),
+                                  p.obs + ((long long)n * 4 + c) * p.in_plane + (long long)Y * strip,
+                                  (uint32_t)(cnt * strip), raw_bar);
+                    R = Re + 1;
+                }
+            };
+            if (pw < n_mma && pw < my_tiles && elect_one()) fetch(t);
+            __syncwarp();
+            int k = 0;  // steps done by this warp
+            for (int i = pw; i < my_tiles && ok && pw < n_mma; i += n_mma, t += n_mma * gridDim.x, ++k) {
+                const int s = pw;  // one stage per ring
+                ok = mbar_wait(empty0 + 8 * s, (uint32_t)((k & 1) ^ 1), abort_flag, p.status, 1);
+                if (ok) ok = mbar_wait(raw_bar, (uint32_t)(k & 1), abort_flag, p.status, 32);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const long long g0 = (long long)t * kTileM * SUB;
+                const int x0 = (int)(g0 % Ws);
+                uint8_t *tile = stages + (size_t)s * stage_bytes;
+                if (p.ingest_clamp == 2) convert_tile<2>(p, raw, tile, g0, x0, total_rows, lane);
+                else if (p.ingest_clamp) convert_tile<1>(p, raw, tile, g0, x0, total_rows, lane);
+                else convert_tile<0>(p, raw, tile, g0, x0, total_rows, lane);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(full0 + 8 * s);
+                // the issuing warp has read the strips too: fetch the next step's
+                ok = mbar_wait(smem_u32(&bars.conv_done[pw]), (uint32_t)(k & 1), abort_flag, p.status, 64);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (i + n_mma < my_tiles && elect_one()) fetch(t + n_mma * gridDim.x);
+                __syncwarp();
+            }
+        }
         // K-split: every warp serves every tile, with the K groups pw, pw + n_mma, ...
         const int tile_step = ksplit ? 1 : n_mma, g_first = ksplit ? pw : 0, g_step = ksplit ? n_mma : 1;
         const int my_groups = g_first < n_groups ? (n_groups - g_first + g_step - 1) / g_step : 0;
         if (ksplit) t = blockIdx.x;
-        for (int i = ksplit ? 0 : pw; i < my_tiles && ok && pw < n_mma; i += tile_step, t += tile_step * gridDim.x) {
+        for (int i = ksplit ? 0 : pw; !FUSE && i < my_tiles && ok && pw < n_mma; i += tile_step, t += tile_step * gridDim.x) {
             int mt = t, nt = 0;
             if (p.n_tiles != 1) {
                 mt = t / p.n_tiles;
@@ -717,6 +843,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 const int s = mw + n_mma * sl;
                 const int j = gi * G;
+                if constexpr (FUSE) {
+                    // build the step's second operand tile (see the producer role)
+                    const int kf = (i - mw) / n_mma;  // steps this warp has done
+                    const int raw_bytes = (4 * p.raw_rows * 4 * p.in_w + 127) & ~127;
+                    const uint8_t *raw = stages + (size_t)n_stages * stage_bytes + (size_t)mw * raw_bytes;
+                    ok = mbar_wait(empty0 + 8 * s, par ^ 1, abort_flag, p.status, 1);
+                    if (ok) ok = mbar_wait(smem_u32(&bars.raw_full[mw]), (uint32_t)(kf & 1), abort_flag, p.status, 32);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    const int step = (int)blockIdx.x + i * (int)gridDim.x;
+                    const long long g0 = (long long)step * kTileM * SUB;
+                    const long long total_rows = (long long)p.batch * p.rows_per_image;
+                    const int x0 = (int)(g0 % p.grid_w);
+                    uint8_t *tile = stages + (size_t)s * stage_bytes;
+                    for (int sub = 1; sub < SUB; ++sub) {
+                        uint8_t *box = tile + sub * box_bytes;
+                        if (p.ingest_clamp == 2)
+                            convert_tile<2>(p, raw, box, g0 + sub * kTileM, x0 + sub * kTileM, total_rows, lane);
+                        else if (p.ingest_clamp)
+                            convert_tile<1>(p, raw, box, g0 + sub * kTileM, x0 + sub * kTileM, total_rows, lane);
+                        else
+                            convert_tile<0>(p, raw, box, g0 + sub * kTileM, x0 + sub * kTileM, total_rows, lane);
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bars.conv_done[mw]));
+                }
                 {
                     TRACE_T0();
                     ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8);
@@ -872,7 +1025,8 @@ size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
     const size_t stage = p.shifted ? p.sub * (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
                                    : (size_t)p.group * (a_chunk + (resident_b ? 0 : b_tile));
-    return 1024 + res + (size_t)p.n_stages * stage + (p.staged ? (size_t)4 * kEpiGroups * kStagingBytes : 0);
+    const size_t raw = p.fuse_ingest ? (size_t)kProdWarps * ((4 * p.raw_rows * 4 * p.in_w + 127) & ~127) : 0;
+    return 1024 + res + (size_t)p.n_stages * stage + (p.staged ? (size_t)4 * kEpiGroups * kStagingBytes : 0) + raw;
 }
 
 static int pow2_floor(int v)
@@ -952,10 +1106,17 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
     cudaError_t e;
     if (p.px_per_row) {
         if (!resident_b || !p.fast_div || p.logits_mode) return cudaErrorInvalidValue;
-        e = extras ? go(tc_gemm_kernel<true, true, true>) : go(tc_gemm_kernel<true, false, true>);
+        e = extras ? go(tc_gemm_kernel<true, true, true, false>) : go(tc_gemm_kernel<true, false, true, false>);
     } else {
-        e = resident_b ? (extras ? go(tc_gemm_kernel<true, true, false>) : go(tc_gemm_kernel<true, false, false>))
-                       : (extras ? go(tc_gemm_kernel<false, true, false>) : go(tc_gemm_kernel<false, false, false>));
+        if (p.fuse_ingest) {
+            if (!resident_b || extras || !p.shifted || p.n_stages != p.n_mma) return cudaErrorInvalidValue;
+            e = go(tc_gemm_kernel<true, false, false, true>);
+        } else {
+            e = resident_b ? (extras ? go(tc_gemm_kernel<true, true, false, false>)
+                                     : go(tc_gemm_kernel<true, false, false, false>))
+                           : (extras ? go(tc_gemm_kernel<false, true, false, false>)
+                                     : go(tc_gemm_kernel<false, false, false, false>));
+        }
     }
     if (e != cudaSuccess) return e;
     return cudaGetLastError();

@@ -77,6 +77,17 @@ struct TcGemmParams {
     int logits_mode;  // 1: write fp32 logits [batch][n_actions] to `logits` instead of int8
     float *logits;
     int n_actions;
+    // fuse_ingest = 1 (first conv on 4-channel uint8 frames stored space-to-depth(4), shifted mode,
+    // one shared-memory stage per issuing warp): no quantised input tensor exists; the producer
+    // warp and the issuing warp of a ring read the raw NCHW frames `obs`, quantise them with
+    // q = min((u * ingest_mul + ingest_add) >> 24, 127) and build the operand tiles of a step in
+    // shared memory themselves.  in_w = frame width, in_plane = bytes of a channel plane,
+    // raw_rows = rows of the input grid a step can touch.
+    int fuse_ingest;
+    const uint8_t *obs;
+    int in_w, in_plane, raw_rows;
+    uint32_t ingest_mul, ingest_add;
+    int ingest_clamp;  // 0: the line never exceeds 127 for u <= 255, the min is left out; 2: the table is u >> 1
     int *status;
     int trace_slot;  // which block of trace counters a traced build adds to
 };

@@ -425,7 +425,35 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             g.shifted = 0;  // fall back to one box per tap
             g.a_rows = 128;
         }
-        if (!tc_choose_pipeline(g, ts.resident_b)) {
+        // The input stage runs inside the first conv when the frames have the shape the fused
+        // producer is written for (4 channels, space-to-depth 4, 16-byte aligned strips) and the
+        // quantiser is the fixed-point line; the parity tap of the quantised input needs the
+        // separate launch.
+        const bool fuse = i == 0 && d.kind == ACCERL_CONV2D && !(p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) &&
+                          p->in_c == 4 && d.stride == 4 && g.chunk_bytes == 64 && g.shifted && ts.resident_b &&
+                          p->ingest_arith == 1 && p->in_w % 4 == 0 && (p->in_h * p->in_w) % 16 == 0 && n_layers > 1;
+        if (fuse) {
+            TcGemmParams f = g;
+            f.fuse_ingest = 1;
+            f.max_sub = 2;
+            f.in_w = p->in_w;
+            f.in_plane = p->in_h * p->in_w;
+            f.raw_rows = (f.grid_w - 1 + 128 + f.a_rows - 1) / f.grid_w + 1;  // two tiles per step
+            f.ingest_mul = p->ingest_mul;
+            f.ingest_add = p->ingest_add;
+            f.ingest_clamp = 0;
+            for (unsigned u = 0; u < 256; ++u)
+                if (((unsigned long long)u * p->ingest_mul + p->ingest_add) >> 24 > 127) f.ingest_clamp = 1;
+            if (p->ingest_shift1) f.ingest_clamp = 2;
+            f.fuse_ingest = 0;  // the ordinary pipeline first: tiles per step, accumulators, issuing warps
+            if (tc_choose_pipeline(f, true)) {
+                f.fuse_ingest = 1;
+                f.n_stages = f.n_mma;  // one stage per ring; the freed room holds the raw strips
+                f.raw_rows = (f.grid_w - 1 + (f.sub - 1) * 128 + f.a_rows - 1) / f.grid_w + 1;
+                if (tc_smem_bytes(f, true) <= 216 * 1024) g = f;
+            }
+        }
+        if (!g.fuse_ingest && !tc_choose_pipeline(g, ts.resident_b)) {
             ts.resident_b = false;
             g.shifted = 0;
             g.a_rows = 128;
@@ -453,6 +481,11 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
         if (g.fast_div) s.kernel += "[3-step divide verified]";
         s.covers = "layer " + std::to_string(i);
+        if (g.fuse_ingest) {  // takes the place of the ingest launch
+            s.kernel += "[frames quantised inside]";
+            s.covers = "ingest+layer 0";
+            steps.clear();
+        }
         steps.push_back(s);
     }
     if (!fused_sample) {
