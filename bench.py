@@ -104,9 +104,12 @@ def algorithmic(name: str, batch: int) -> dict:
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch / states of that launch, from
-# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 188.81 MB read + 127.30 MB written)
+# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 173.51 MB read + 48.45 MB written by the
+# first conv with the input stage inside)
 NCU_DRAM_BYTES_PER_STATE = {
-    ("nature_cnn_b8192", "ingest_u8_s2d44_kernel"): (188809216 + 127298560) / 6144,
+    ("nature_cnn_b8192",
+     "tc_gemm_kernel<resident weights>[3-step divide verified][frames quantised inside]"):
+        (173507328 + 48445440) / 6144,
 }
 
 
