@@ -304,14 +304,14 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut,
                                                    p->bufs[p->layers[0].in_buf].ptr, B, p->in_h,
                                                    p->in_w, p->in_h, p->in_w, 0, 0,
-                                                   p->ingest_float ? 2 : p->ingest_arith,
+                                                   p->ingest_shift1 ? 4 : (p->ingest_float ? 2 : p->ingest_arith),
                                                    p->ingest_float ? p->ingest_fa : p->ingest_mul,
                                                    p->ingest_float ? p->ingest_fc1 : p->ingest_add, st));
             break;
         case Step::INGEST_PAD4:
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut, p->in_pad4, B,
                                                    p->in_h, p->in_w, p->in_h + 2, p->in_pad4_w, 1, 4,
-                                                   p->ingest_float ? 2 : p->ingest_arith,
+                                                   p->ingest_shift1 ? 4 : (p->ingest_float ? 2 : p->ingest_arith),
                                                    p->ingest_float ? p->ingest_fa : p->ingest_mul,
                                                    p->ingest_float ? p->ingest_fc1 : p->ingest_add, st));
             break;

@@ -109,6 +109,10 @@ __global__ void ingest_u8_nhwc4_kernel(const uint8_t *__restrict__ obs, const in
     for (int c = 0; c < 4; ++c)
         plane[c] = __ldg(reinterpret_cast<const uint32_t *>(obs + ((n * 4 + c) * H + y) * W) + x4);
     uint32_t w[4];
+    if (ARITH == 4) {  // the table is u >> 1: four bytes at a time, then a 4 x 4 byte transpose
+        const uint4 v = ingest_shift_line16(plane[0], plane[1], plane[2], plane[3]);
+        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+    } else
 #pragma unroll
     for (int px = 0; px < 4; ++px) {
         if (ARITH == 2) {
@@ -139,7 +143,10 @@ cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t
 {
     const long long total = (long long)B * H * (W / 4);
     const unsigned blocks = (unsigned)((total + 255) / 256);
-    if (arith == 2)
+    if (arith == 4)
+        ingest_u8_nhwc4_kernel<4><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
+                                                         out_wpitch, off_y, off_x, mul, add);
+    else if (arith == 2)
         ingest_u8_nhwc4_kernel<2><<<blocks, 256, 0, st>>>(obs, lut, out, total, H, W / 4, out_hpitch,
                                                          out_wpitch, off_y, off_x, mul, add);
     else if (arith == 1)
