@@ -499,17 +499,19 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
     }
 }
 
-// Fused input stage: one operand tile (a_rows rows from GEMM row g0 on) from the raw frame strips
+// Fused input stage: rows [row_begin, row_end) of a step's operand rows (from GEMM row g0 on;
+// the tiles of a step are 128 rows apart in one contiguous block) from the raw frame strips
 // in shared memory, one lane per row: sixteen 4-byte loads (4 image rows x 4 channel planes), 64
 // quantised bytes in (dy, dx, c) order, stored as four 16-byte pieces under the 64-byte swizzle
 // (piece index XOR address bits 7..8).  Rows past the last state are zero.  t0 = position of g0
 // relative to the first column of the first grid row held in `raw`.
 template <int MODE>  // 0: line without the min, 1: line with it, 2: q = u >> 1
 __device__ __forceinline__ void convert_tile(const TcGemmParams &p, const uint8_t *raw, uint8_t *tile,
-                                             long long g0, int t0, long long total_rows, int lane)
+                                             long long g0, int t0, long long total_rows, int row_begin,
+                                             int row_end, int lane)
 {
     const int Ws = p.grid_w, strip = 4 * p.in_w;
-    for (int rr = lane; rr < p.a_rows; rr += 32) {
+    for (int rr = row_begin + lane; rr < row_end; rr += 32) {
         const unsigned tt = (unsigned)(t0 + rr);
         const int Rrel = (int)__umulhi(tt, p.grid_w_magic), X = (int)tt - Rrel * Ws;
         uint4 q[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0),
@@ -582,8 +584,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // sub > 1 (shifted mode only): a pipeline step covers `sub` consecutive 128-row tiles, one TMA
     // box and one accumulator each, so that the barrier round trips are paid once per step
     const int SUB = p.sub;
-    const int box_bytes = (p.a_rows * CH + 1023) & ~1023;
-    const int stage_bytes = p.shifted ? SUB * box_bytes
+    // (fused input stage: the tiles of a step overlap in one contiguous block of rows)
+    const int box_bytes = FUSE ? kTileM * CH : (p.a_rows * CH + 1023) & ~1023;
+    const int stage_bytes = FUSE ? ((((SUB - 1) * kTileM + p.a_rows) * CH + 1023) & ~1023)
+                            : p.shifted ? SUB * box_bytes
                                       : p.group * (a_chunk_bytes + (RESIDENT_B ? 0 : b_tile_bytes));
     uint8_t *resident_b = smem;
     uint8_t *stages = smem + (RESIDENT_B ? ((p.n_chunks * b_tile_bytes + 1023) & ~1023) : 0);
@@ -731,9 +735,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const long long g0 = (long long)t * kTileM * SUB;
                 const int x0 = (int)(g0 % Ws);
                 uint8_t *tile = stages + (size_t)s * stage_bytes;
-                if (p.ingest_clamp == 2) convert_tile<2>(p, raw, tile, g0, x0, total_rows, lane);
-                else if (p.ingest_clamp) convert_tile<1>(p, raw, tile, g0, x0, total_rows, lane);
-                else convert_tile<0>(p, raw, tile, g0, x0, total_rows, lane);
+                // this warp converts the first rows of the step, the ring's issuing warp the rest
+                const int split = SUB > 1 ? ((step_rows / 2 + 31) & ~31) : step_rows;
+                if (p.ingest_clamp == 2) convert_tile<2>(p, raw, tile, g0, x0, total_rows, 0, split, lane);
+                else if (p.ingest_clamp) convert_tile<1>(p, raw, tile, g0, x0, total_rows, 0, split, lane);
+                else convert_tile<0>(p, raw, tile, g0, x0, total_rows, 0, split, lane);
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(full0 + 8 * s);
@@ -857,15 +863,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const long long total_rows = (long long)p.batch * p.rows_per_image;
                     const int x0 = (int)(g0 % p.grid_w);
                     uint8_t *tile = stages + (size_t)s * stage_bytes;
-                    for (int sub = 1; sub < SUB; ++sub) {
-                        uint8_t *box = tile + sub * box_bytes;
-                        if (p.ingest_clamp == 2)
-                            convert_tile<2>(p, raw, box, g0 + sub * kTileM, x0 + sub * kTileM, total_rows, lane);
-                        else if (p.ingest_clamp)
-                            convert_tile<1>(p, raw, box, g0 + sub * kTileM, x0 + sub * kTileM, total_rows, lane);
-                        else
-                            convert_tile<0>(p, raw, box, g0 + sub * kTileM, x0 + sub * kTileM, total_rows, lane);
-                    }
+                    const int step_rows = (SUB - 1) * kTileM + p.a_rows;
+                    const int split = SUB > 1 ? ((step_rows / 2 + 31) & ~31) : step_rows;
+                    if (p.ingest_clamp == 2) convert_tile<2>(p, raw, tile, g0, x0, total_rows, split, step_rows, lane);
+                    else if (p.ingest_clamp) convert_tile<1>(p, raw, tile, g0, x0, total_rows, split, step_rows, lane);
+                    else convert_tile<0>(p, raw, tile, g0, x0, total_rows, split, step_rows, lane);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&bars.conv_done[mw]));
@@ -1023,7 +1025,9 @@ size_t tc_smem_bytes(const TcGemmParams &p, bool resident_b)
 {
     const int a_chunk = kTileM * p.chunk_bytes, b_tile = p.n_tile * (p.kstep_list ? 32 : p.chunk_bytes);
     size_t res = resident_b ? (((size_t)p.n_chunks * b_tile + 1023) & ~(size_t)1023) : 0;
-    const size_t stage = p.shifted ? p.sub * (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
+    const size_t stage = p.fuse_ingest
+                             ? ((((size_t)(p.sub - 1) * kTileM + p.a_rows) * p.chunk_bytes + 1023) & ~(size_t)1023)
+                         : p.shifted ? p.sub * (((size_t)p.a_rows * p.chunk_bytes + 1023) & ~(size_t)1023)
                                    : (size_t)p.group * (a_chunk + (resident_b ? 0 : b_tile));
     const size_t raw = p.fuse_ingest ? (size_t)kProdWarps * ((4 * p.raw_rows * 4 * p.in_w + 127) & ~127) : 0;
     return 1024 + res + (size_t)p.n_stages * stage + (p.staged ? (size_t)4 * kEpiGroups * kStagingBytes : 0) + raw;
