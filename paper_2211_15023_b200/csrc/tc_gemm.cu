@@ -689,9 +689,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // frames, R = image * grid_h + Y.  The four image rows 4Y .. 4Y+3 of one channel are
             // in_w * 4 contiguous, 16-byte aligned bytes and consecutive Y of an image follow each
             // other, so the raw bytes under a step arrive with at most two bulk copies per channel
-            // plane.  This warp then builds the step's first operand tile, the ring's issuing warp
-            // the second (or the upper half of a single one); both fence their writes to the async
-            // proxy.  The ring has one stage and one raw buffer: the next step's strips are fetched
+            // plane.  This warp then builds the first half of the step's operand rows (the tiles of
+            // a step are 128 rows apart in one contiguous block), the ring's issuing warp the second
+            // half; both fence their writes to the async proxy.  The ring has one stage and one raw
+            // buffer: the next step's strips are fetched
             // as soon as both warps have read the current ones, while the MMAs of this step run.
             const int Ws = p.grid_w, Hs = p.rows_per_image / Ws, strip = 4 * p.in_w;
             const long long total_rows = (long long)p.batch * p.rows_per_image;
