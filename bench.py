@@ -104,12 +104,12 @@ def algorithmic(name: str, batch: int) -> dict:
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch / states of that launch, from
-# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 173.51 MB read + 48.45 MB written by the
+# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 173.52 MB read + 48.61 MB written by the
 # first conv with the input stage inside)
 NCU_DRAM_BYTES_PER_STATE = {
     ("nature_cnn_b8192",
      "tc_gemm_kernel<resident weights>[3-step divide verified][frames quantised inside]"):
-        (173507328 + 48445440) / 6144,
+        (173518848 + 48606464) / 6144,
 }
 
 
