@@ -224,6 +224,23 @@ def test_tensor_core_logits_layer_with_many_actions():
         g.close()
 
 
+@pytest.mark.parametrize("name", ["nature_cnn_b160", "student_cnn_b8192"])
+def test_input_stage_inside_first_conv_small_and_ragged_batches(name):
+    """Without the parity taps the frames are quantised inside the first conv (no launch of their
+    own): batches from one state up, none a multiple of the 256 GEMM rows of a pipeline step."""
+    import paper_2211_15023_b200 as P
+    pol = calibrated(name)
+    g = P.Policy(pol, 61, flags=0)
+    assert "frames quantised inside" in g.info()["plan"]
+    for b in (1, 2, 5, 37, 61):
+        obs, u = W.observations(name, b, seed=77 + b), W.uniforms(name, b, seed=78 + b)
+        ref = oracle.forward(pol, obs, u, keep=False)
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        g.check()
+        compare(ref, *out)
+    g.close()
+
+
 def test_exact_ties_on_the_tensor_core_path():
     """Power-of-two scales make many epilogue quotients land exactly on k + 0.5: the requantiser
     must round them to even exactly as the IEEE divide + rintf of the definition does."""
