@@ -5,8 +5,9 @@ import this package.  It shares no code with the CUDA library and never
 imports it.  ``accerl_oracle.c`` holds the arithmetic (naive loops), this
 package compiles it with gcc, loads it through ctypes and composes the
 per-layer calls into a whole forward pass (``forward``), a post-training
-quantiser and calibrator (``ptq``).
+quantiser and calibrator (``ptq``); ``corrector`` wraps the V-trace definition.
 """
 from .clib import build, lib  # noqa: F401
-from .net import forward, ingest, layer_acc, layer_float  # noqa: F401
+from .corrector import vtrace  # noqa: F401
+from .net import entropy, forward, forward_mixed, ingest, kl, layer_acc, layer_float  # noqa: F401
 from .ptq import calibrate, prune_2_4, quantise_weights  # noqa: F401

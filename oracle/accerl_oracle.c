@@ -29,7 +29,8 @@
  * Parity status: every function below is pinned by the CPU tests (hand-worked
  * two-layer example, fp64 de-quantised forward, float64 library convolutions
  * on integer tensors, structural special cases, brute force for the sampler,
- * exhaustive ingest).  What stays unpinned: that this quantisation scheme is
+ * exhaustive ingest; entropy and KL against closed forms and scipy; V-trace
+ * against the n-step return, the one-step TD target and a hand-worked rollout).  What stays unpinned: that this quantisation scheme is
  * the one the paper's authors ran -- the paper says only "PTQ" and "int8".
  */
 #include <math.h>
@@ -202,5 +203,110 @@ void oracle_sample(const float *logits, int B, int A, const float *u, double *lo
         action[n] = a;
         logp_a[n] = (float)lp[a];
         margin[n] = best;
+    }
+}
+
+/*
+ * Entropy of the action distribution, H(pi(.|s)) = -sum_i p_i log p_i, per state, in double
+ * from the fp32 logits.  The paper uses it twice: as the regulariser of the distillation loss
+ * (Section 2.2, Eq. KD, the term -beta H(pi_smaller)) and as one of the Monitor's indicators
+ * (Section 2.4; Eq. advance lists "entropy" among the strategy's inputs).  Terms with p_i = 0
+ * (exp underflow) contribute 0.
+ */
+void oracle_entropy(const float *logits, int B, int A, double *h)
+{
+#pragma omp parallel for
+    for (int n = 0; n < B; ++n) {
+        const float *z = logits + (int64_t)n * A;
+        double m = (double)z[0];
+        for (int i = 1; i < A; ++i)
+            if ((double)z[i] > m) m = (double)z[i];
+        double s = 0.0;
+        for (int i = 0; i < A; ++i) s += exp((double)z[i] - m);
+        const double lse = m + log(s);
+        double acc = 0.0;
+        for (int i = 0; i < A; ++i) {
+            const double lp = (double)z[i] - lse, p = exp(lp);
+            if (p > 0.0) acc -= p * lp;
+        }
+        h[n] = acc;
+    }
+}
+
+/*
+ * KL(pi_original || pi_smaller) = sum_a pi_original(a|x) log(pi_original(a|x) / pi_smaller(a|x))
+ * per state (Section 2.4, Eq. KL: the Monitor's "KL mean" / "KL max" indicators are the mean and
+ * the maximum of this over a batch), in double from two fp32 logit rows.
+ */
+void oracle_kl(const float *logits_original, const float *logits_smaller, int B, int A, double *kl)
+{
+#pragma omp parallel for
+    for (int n = 0; n < B; ++n) {
+        const float *zo = logits_original + (int64_t)n * A, *zs = logits_smaller + (int64_t)n * A;
+        double mo = (double)zo[0], ms = (double)zs[0];
+        for (int i = 1; i < A; ++i) {
+            if ((double)zo[i] > mo) mo = (double)zo[i];
+            if ((double)zs[i] > ms) ms = (double)zs[i];
+        }
+        double so = 0.0, ss = 0.0;
+        for (int i = 0; i < A; ++i) {
+            so += exp((double)zo[i] - mo);
+            ss += exp((double)zs[i] - ms);
+        }
+        const double lseo = mo + log(so), lses = ms + log(ss);
+        double acc = 0.0;
+        for (int i = 0; i < A; ++i) {
+            const double lpo = (double)zo[i] - lseo, lps = (double)zs[i] - lses, p = exp(lpo);
+            if (p > 0.0) acc += p * (lpo - lps);
+        }
+        kl[n] = acc;
+    }
+}
+
+/*
+ * V-trace targets (Section 2.3, Eq. V-trace), written out as the definition: for every start
+ * step s of a rollout of n steps,
+ *
+ *   v_s     = V(x_s) + sum_{t=s}^{n-1} (prod_{i=s}^{t-1} g_i c_i) delta_t
+ *   delta_t = rho_t (r_t + g_t V(x_{t+1}) - V(x_t))
+ *   rho_t   = min(rho_hat, pi_original / pi_smaller),   c_i = min(c_hat, pi_original / pi_smaller)
+ *
+ * with pi_original / pi_smaller = exp(logp_original - logp_smaller) of the action taken and
+ * V(x_n) = bootstrap.  g_t is the constant gamma of the equation, or discounts[t] when a
+ * per-step array is given (gamma times "episode goes on", the usual way of cutting the sums at
+ * an episode end inside a rollout).  The sum of start step s runs to the end of the rollout.
+ * Also returns the policy-gradient advantage of Eq. A3C-V's first line,
+ *   adv_s = rho_s (r_s + g_s v_{s+1} - V(x_s)),  v_n = V(x_n).
+ * All arrays are time-major [n][B]; everything is computed in double.
+ */
+void oracle_vtrace(const float *logp_smaller, const float *logp_original, const float *rewards,
+                   const float *values, const float *bootstrap, const float *discounts, int n,
+                   int B, float gamma, float rho_hat, float c_hat, double *vs, double *adv)
+{
+#pragma omp parallel for
+    for (int b = 0; b < B; ++b) {
+        for (int s = 0; s < n; ++s) {
+            double sum = 0.0, prod = 1.0;
+            for (int t = s; t < n; ++t) {
+                const int64_t i = (int64_t)t * B + b;
+                const double ratio = exp((double)logp_original[i] - (double)logp_smaller[i]);
+                const double rho = ratio < (double)rho_hat ? ratio : (double)rho_hat;
+                const double c = ratio < (double)c_hat ? ratio : (double)c_hat;
+                const double g = discounts ? (double)discounts[i] : (double)gamma;
+                const double v_next = t + 1 < n ? (double)values[i + B] : (double)bootstrap[b];
+                const double delta = rho * ((double)rewards[i] + g * v_next - (double)values[i]);
+                sum += prod * delta;
+                prod *= g * c;
+            }
+            vs[(int64_t)s * B + b] = (double)values[(int64_t)s * B + b] + sum;
+        }
+        for (int s = 0; s < n; ++s) {
+            const int64_t i = (int64_t)s * B + b;
+            const double ratio = exp((double)logp_original[i] - (double)logp_smaller[i]);
+            const double rho = ratio < (double)rho_hat ? ratio : (double)rho_hat;
+            const double g = discounts ? (double)discounts[i] : (double)gamma;
+            const double v_next = s + 1 < n ? vs[i + B] : (double)bootstrap[b];
+            adv[i] = rho * ((double)rewards[i] + g * v_next - (double)values[i]);
+        }
     }
 }

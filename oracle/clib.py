@@ -29,6 +29,7 @@ def lib() -> ctypes.CDLL:
         _lib = ctypes.CDLL(build())
         for name in ("oracle_ingest_u8", "oracle_ingest_f32", "oracle_conv_acc", "oracle_fc_acc",
                      "oracle_skip_add", "oracle_epilogue_float", "oracle_requant",
-                     "oracle_maxpool", "oracle_sample"):
+                     "oracle_maxpool", "oracle_sample", "oracle_entropy", "oracle_kl",
+                     "oracle_vtrace"):
             getattr(_lib, name).restype = None
     return _lib

@@ -99,14 +99,38 @@ def sample(logits: np.ndarray, u: np.ndarray) -> dict:
     return dict(logp_all=logp_all, actions=actions, logp=logp, margin=margin)
 
 
+def entropy(logits: np.ndarray) -> np.ndarray:
+    """Per-state entropy of softmax(logits), float64."""
+    logits = np.ascontiguousarray(logits, np.float32)
+    b, a = logits.shape
+    h = np.empty(b, np.float64)
+    lib().oracle_entropy(_p(logits), b, a, _p(h))
+    return h
+
+
+def kl(logits_original: np.ndarray, logits_smaller: np.ndarray) -> np.ndarray:
+    """Per-state KL(pi_original || pi_smaller) from two logit matrices, float64."""
+    lo = np.ascontiguousarray(logits_original, np.float32)
+    ls = np.ascontiguousarray(logits_smaller, np.float32)
+    assert lo.shape == ls.shape
+    b, a = lo.shape
+    out = np.empty(b, np.float64)
+    lib().oracle_kl(_p(lo), _p(ls), b, a, _p(out))
+    return out
+
+
 def forward(policy: dict, obs: np.ndarray, u: np.ndarray, keep: bool = True) -> dict:
-    """Forward + sampling.  Returns logits, actions, logp, logp_all, margin and, with
-    ``keep``, ``input_q`` and ``activations`` (one int8 NCHW array per non-final layer)."""
+    """Forward + sampling.  Returns logits, actions, logp, logp_all, margin, entropy and, with
+    ``keep``, ``input_q`` and ``activations`` (one int8 NCHW array per non-final layer).
+
+    A final layer with ``value`` set has one output column more than there are actions: that
+    last column is the state value V(s) (the same single fma as a logit, no requantisation);
+    it is returned as ``value`` and takes no part in the softmax."""
     b = obs.shape[0]
     x = ingest(policy["in_kind"], obs, policy["s_input"]).reshape((b,) + tuple(policy["in_shape"]))
     outs = []
     input_q = x
-    logits = None
+    logits = value = None
     for l in policy["layers"]:
         if l["kind"] == "maxpool":
             x = maxpool(l, x)
@@ -117,13 +141,35 @@ def forward(policy: dict, obs: np.ndarray, u: np.ndarray, keep: bool = True) -> 
             y = layer_float(l, acc)
             if l["logits"]:
                 logits = y.reshape(b, -1)
+                if l.get("value"):
+                    value = np.ascontiguousarray(logits[:, -1])
+                    logits = np.ascontiguousarray(logits[:, :-1])
                 outs.append(None)
                 break
             x = requant(y, l["s_out"])
         outs.append(x)
     res = sample(logits, u)
     res["logits"] = logits
+    res["entropy"] = entropy(logits)
+    if value is not None:
+        res["value"] = value
     if keep:
         res["input_q"] = input_q
         res["activations"] = outs
     return res
+
+
+def forward_mixed(smaller: dict, original: dict, obs: np.ndarray, u: np.ndarray,
+                  u_select: np.ndarray, alpha: float) -> dict:
+    """Per-state choice between two policies: state i runs ``smaller`` when
+    ``u_select[i] < alpha`` and ``original`` otherwise (the Actor uses the small network with
+    probability alpha).  Returns the chosen network's outputs per state plus ``use_smaller``."""
+    rs = forward(smaller, obs, u, keep=False)
+    ro = forward(original, obs, u, keep=False)
+    pick = np.asarray(u_select, np.float32) < np.float32(alpha)
+    out = dict(use_smaller=pick)
+    for k in ("logits", "actions", "logp", "logp_all", "margin", "entropy", "value"):
+        if k in rs and k in ro:
+            sel = pick.reshape((-1,) + (1,) * (rs[k].ndim - 1))
+            out[k] = np.where(sel, rs[k], ro[k])
+    return out

@@ -31,9 +31,18 @@ def _conv(in_c, in_h, in_w, out_c, k, stride, pad, relu_in=False, relu_out=True,
                 skip_from=skip_from)
 
 
-def _fc(k, n, relu_in=False, relu_out=True, logits=False):
+def _fc(k, n, relu_in=False, relu_out=True, logits=False, value=False):
     return dict(kind="fc", in_c=k, in_h=1, in_w=1, out_c=n, kh=1, kw=1, stride=1, pad=0,
-                relu_in=relu_in, relu_out=relu_out, logits=logits, skip_from=-1)
+                relu_in=relu_in, relu_out=relu_out, logits=logits, skip_from=-1, value=value)
+
+
+def with_value_head(layers: List[dict]) -> List[dict]:
+    """The same architecture with a state-value output: the last layer gets one more output
+    column (the value V(s)) after its action logits."""
+    out = [dict(l) for l in layers]
+    out[-1]["out_c"] += 1
+    out[-1]["value"] = True
+    return out
 
 
 def _pool(c, h, w, k=3, stride=2):
