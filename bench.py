@@ -97,9 +97,13 @@ class ClockSampler:
 
 
 def algorithmic(name: str, batch: int) -> dict:
-    """Algorithmic work of one step: 2 x MACs, and input + output bytes per state."""
+    """Algorithmic work of one step: 2 x useful MACs, and input + output bytes per state.
+
+    For a 2:4-pruned workload half of the dense MACs multiply structural zeros and are no
+    algorithmic work; `ops_dense_executed` is what a dense contraction still performs."""
     a = W.n_actions(name)
-    return dict(ops=2 * W.macs_per_state(name) * batch,
+    dense = 2 * W.macs_per_state(name) * batch
+    return dict(ops=dense // 2 if W.config(name)["prune24"] else dense, ops_dense_executed=dense,
                 bytes=(W.input_bytes_per_state(name) + 4 + OUT_BYTES(a)) * batch)
 
 
@@ -246,7 +250,11 @@ def time_workload(P, torch, name, batch, steps, warmup, n_buffers, device, dist=
     for i in range(steps):
         per += g.act_timed(obs[i % n_buffers], u, out, stream.cuda_stream)
     per /= steps
+    # one more step on the un-rotated batch, outside every timed region: what the parity check reads
+    g.act(obs[0], u, out, stream.cuda_stream)
+    torch.cuda.synchronize()
     res = dict(ms=ms, info=info, per_launch_ms=per, policy=g, obs=obs_np, u=u, out=out,
+               check_out=tuple(t.cpu().numpy() for t in out),
                clocks=sampler.summary() if sampler else None)
     return res
 
@@ -292,6 +300,7 @@ def main() -> None:
     ms = r["ms"]
     g = r["policy"]
     clocks = r["clocks"]
+    check_out = r["check_out"]
     value = job_value(batch, world, ms)
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies timed)
@@ -365,22 +374,37 @@ def main() -> None:
             floor = max(w["ops"] / (int8_peak * 1e12), w["bytes"] / (pk["hbm_gbs"] * 1e9)) * 1e3
             others[other] = dict(batch=ob, ms_per_step=o["ms"], states_per_s=ob / (o["ms"] * 1e-3),
                                  launches=o["info"]["launches_per_act"],
+                                 ops_per_state=w["ops"] // ob,
+                                 ops_per_state_dense_executed=w["ops_dense_executed"] // ob,
                                  frac_of_step_roofline=floor / o["ms"])
             o["policy"].close()
 
     # ---- CPU oracle on a bounded sample of the same workload (reported baseline)
-    cpu = None
+    # and the parity of what was timed: the GPU outputs of those states (same policy, same plan,
+    # full batch) against the oracle's, outside the timed region
+    cpu = parity = None
     if not args.no_cpu:
         import oracle
         sample = min(batch, args.cpu_sample)
         pol = W.drawn_int8_policy(name)
-        so, su = W.observations(name, sample), W.uniforms(name, sample)
+        so, su = W.observations(name, batch)[:sample], W.uniforms(name, batch)[:sample]
         oracle.forward(pol, so[:8], su[:8], keep=False)
         t0 = time.perf_counter()
-        oracle.forward(pol, so, su, keep=False)
+        ref = oracle.forward(pol, so, su, keep=False)
         cpu_dt = time.perf_counter() - t0
         cpu = dict(value=sample / cpu_dt, unit=UNIT, cores=os.cpu_count(), kind="oracle",
                    sample="first %d states of the %d-state batch, one pass" % (sample, batch))
+        lg, ac, lp = (a[:sample] for a in check_out)
+        diff = ac != ref["actions"]
+        same = ~diff
+        lp_err = np.abs(lp[same].astype(np.float64) - ref["logp"][same])
+        lp_tol = 1e-6 + 1e-5 * np.abs(ref["logp"][same])
+        parity = dict(states=int(sample), logits_mismatch=int((lg != ref["logits"]).sum()),
+                      action_mismatch=int(diff.sum()),
+                      action_mismatch_near_edge=int((diff & (ref["margin"] < 1e-5)).sum()),
+                      logp_out_of_tolerance=int((lp_err > lp_tol).sum()),
+                      logp_max_abs_err=float(lp_err.max()) if lp_err.size else 0.0,
+                      note="timed policy and plan, full batch; logits compared bit for bit")
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -398,9 +422,11 @@ def main() -> None:
         "roofline": roof,
         "step_roofline": {"floor_ms": step_floor_ms, "frac": step_floor_ms / ms,
                           "ops_per_state": whole["ops"] // batch,
+                          "ops_per_state_dense_executed": whole["ops_dense_executed"] // batch,
                           "bytes_per_state": whole["bytes"] // batch},
         "launches": launches,
         "cpu_baseline": cpu,
+        "parity": parity,
         "other_workloads": others,
     }
     print(json.dumps(line))

@@ -67,8 +67,15 @@ enum {
 enum {
     ACCERL_FLAG_KEEP_ACTIVATIONS = 1, /* give every layer its own output buffer so that
                                          accerl_policy_read_activation works (parity taps) */
-    ACCERL_FLAG_FORCE_GENERIC = 2     /* use only the plain CUDA-core kernels (no tensor-core
+    ACCERL_FLAG_FORCE_GENERIC = 2,    /* use only the plain CUDA-core kernels (no tensor-core
                                          or fused plans); for cross-checking the fast paths */
+    ACCERL_FLAG_TAP_FUSED = 4         /* only with KEEP_ACTIVATIONS: keep every fusion of the plan
+                                         that runs without the taps (input stage inside the first
+                                         conv, pooling on accumulators, the single-launch MLP) and
+                                         tap the tensors that plan still stores; a tensor it never
+                                         stores reads as ACCERL_ERR_UNSUPPORTED.  Without this
+                                         bit KEEP_ACTIVATIONS un-fuses those steps so that every
+                                         tensor exists. */
 };
 
 /*
@@ -164,13 +171,16 @@ accerl_status accerl_policy_act_timed(accerl_policy *p, const void *obs_dev,
  *
  * Same arguments, ownership and alignment rules as accerl_policy_act, except that `batch` is not
  * limited by the handle's max_batch but by the array: a batch whose activations do not fit is
- * rejected with ACCERL_ERR_BATCH_TOO_LARGE and a message that gives both sizes (Nature-CNN fits
- * about 1400 states).  The call enqueues on `cuda_stream`, returns without synchronising, and calls
+ * rejected with ACCERL_ERR_BATCH_TOO_LARGE and a message that gives both sizes (Nature-CNN, whose
+ * plan reuses two buffers of 28 224 + 12 800 bytes per state, fits about 1600 states).  The call enqueues on `cuda_stream`, returns without synchronising, and calls
  * no cudaMalloc / cudaFree or any other allocating routine.
  *
  * First call on a device: the library asks the CUDA runtime for the array's address on that
  * device (once per device, remembered afterwards).  Make this first call during start-up, before
- * any stream capture is begun.
+ * any stream capture is begun.  The CUDA runtime loads a library's device code lazily, so the
+ * array's memory may only be reserved when this first call (or any earlier kernel of the library
+ * on that device, accerl_policy_create included) triggers the load; on a device without 64 MiB to
+ * spare that is where ACCERL_ERR_CUDA appears.  From the second call on nothing is reserved.
  *
  * Sharing: all handles and all calls in the process use the same array, and it keeps whatever
  * the previous call left in it.  Nothing in it has to start at zero -- every byte a kernel reads
@@ -202,7 +212,9 @@ accerl_status accerl_policy_act_host(accerl_policy *p, const void *obs_host,
  * canonical NCHW order ([batch, out_c, out_h, out_w]; for FC layers [batch, out_c]).
  * `layer` = -1 reads the quantised input tensor ([batch, C, H, W] or [batch, D]).
  * Needs ACCERL_FLAG_KEEP_ACTIVATIONS; synchronises the device.  The final (logits) layer has
- * no int8 output (INVALID_ARG).  dst_bytes must be at least the tensor's size.
+ * no int8 output (INVALID_ARG).  dst_bytes must be at least the tensor's size.  With
+ * ACCERL_FLAG_TAP_FUSED a tensor that the fused plan never stores in un-ReLU'd int8 form gives
+ * ACCERL_ERR_UNSUPPORTED.
  */
 accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int32_t batch,
                                             int8_t *dst_host_nchw, size_t dst_bytes);
@@ -217,7 +229,8 @@ accerl_status accerl_policy_check(accerl_policy *p);
  * Describe the handle: number of actions, bytes of device workspace, kernel launches per
  * `act` call and a human-readable plan (one line per launch) written as a NUL-terminated
  * string into plan_buf (truncated to plan_buf_bytes).  Any output pointer may be NULL.
- * `batch` selects which plan is described (plans can differ by batch size).
+ * The plan is fixed at create time for max_batch; `batch` is accepted for symmetry with the act
+ * calls and does not change the answer.
  */
 accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t *n_actions,
                                  size_t *workspace_bytes, int32_t *launches_per_act,

@@ -7,4 +7,4 @@ is no CPU fallback -- importing :class:`Policy` without the built library
 raises.
 """
 from .binding import (AccerlError, Policy, library, library_path, FLAG_FORCE_GENERIC,  # noqa: F401
-                      FLAG_KEEP_ACTIVATIONS)
+                      FLAG_KEEP_ACTIVATIONS, FLAG_TAP_FUSED)

@@ -11,6 +11,7 @@ _LIB = None
 
 FLAG_KEEP_ACTIVATIONS = 1
 FLAG_FORCE_GENERIC = 2
+FLAG_TAP_FUSED = 4
 RELU_IN, RELU_OUT, LOGITS = 1, 2, 4
 _KINDS = {"conv": 0, "fc": 1, "maxpool": 2}
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "BATCH_TOO_LARGE", 4: "OOM", 5: "CUDA",

@@ -374,8 +374,12 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         set_error("create: n_layers, max_batch and s_input must be positive");
         return ACCERL_ERR_INVALID_ARG;
     }
-    if (flags & ~(uint32_t)(ACCERL_FLAG_KEEP_ACTIVATIONS | ACCERL_FLAG_FORCE_GENERIC)) {
+    if (flags & ~(uint32_t)(ACCERL_FLAG_KEEP_ACTIVATIONS | ACCERL_FLAG_FORCE_GENERIC | ACCERL_FLAG_TAP_FUSED)) {
         set_error("create: unknown flag bits 0x%x", flags);
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    if ((flags & ACCERL_FLAG_TAP_FUSED) && !(flags & ACCERL_FLAG_KEEP_ACTIVATIONS)) {
+        set_error("create: ACCERL_FLAG_TAP_FUSED needs ACCERL_FLAG_KEEP_ACTIVATIONS");
         return ACCERL_ERR_INVALID_ARG;
     }
     // ---- validate the chain on the host before touching the device
@@ -573,6 +577,7 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         p->steps.push_back(ss);
     }
     p->tensor_s2d.assign(n_layers + 1, 1);
+    p->tap_missing.assign(n_layers + 1, 0);
     {
         cudaDeviceProp prop;
         cudaError_t pe = cudaGetDeviceProperties(&prop, device);
@@ -592,7 +597,7 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         if ((st = build_tc_plan(p, layers, n_layers, &used)) != ACCERL_OK) return fail(st);
         if (!used && (st = build_tc_mixed_plan(p, layers, n_layers, &used)) != ACCERL_OK)
             return fail(st);
-        if (!used && !(flags & ACCERL_FLAG_KEEP_ACTIVATIONS) &&
+        if (!used && !unfuse_for_taps(p) &&
             (st = build_mlp_plan(p, layers, n_layers, &used)) != ACCERL_OK)
             return fail(st);
     }
@@ -723,6 +728,10 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
     if (dst_bytes < need) {
         set_error("read_activation: destination holds %zu bytes, %zu needed", dst_bytes, need);
         return ACCERL_ERR_INVALID_ARG;
+    }
+    if (p->tap_missing[layer + 1]) {
+        set_error("read_activation: the fused plan never stores tensor %d", layer);
+        return ACCERL_ERR_UNSUPPORTED;
     }
     DeviceGuard guard(p->device);
     if ((size_t)(layer + 1) < p->taps.size() && p->taps[layer + 1].ptr) {

@@ -122,6 +122,7 @@ struct accerl_policy {
     int8_t *in_pad4 = nullptr;            // frames as [n][H+2][PW][4] with the image at (1, 4)
     int in_pad4_w = 0;
     std::vector<accerl::TapDesc> taps;    // per tensor (index t + 1); empty or null ptr = generic buffer
+    std::vector<char> tap_missing;        // per tensor (index t + 1): the plan never stores it (TAP_FUSED)
     std::shared_ptr<accerl::MlpFusedParams> mlp;  // set when the whole step is one fused launch
     accerl::FcSampleParams fc_sample = {};         // used by a Step::FC_SAMPLE launch
     std::vector<int> tensor_s2d;          // space-to-depth factor of tensor t at [t + 1]
@@ -145,6 +146,12 @@ struct accerl_policy {
 };
 
 namespace accerl {
+
+// KEEP_ACTIVATIONS without TAP_FUSED: build the plan whose every tensor exists
+static inline bool unfuse_for_taps(const accerl_policy *p)
+{
+    return (p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) && !(p->flags & ACCERL_FLAG_TAP_FUSED);
+}
 
 // generic CUDA-core kernels (generic_kernels.cu); every launcher enqueues on `st` and returns
 // the launch status

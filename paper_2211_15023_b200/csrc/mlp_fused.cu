@@ -30,6 +30,10 @@ struct MlpFusedParams {
     const int32_t *w[kMaxLayers];     // [k4][n_pad] words, n_pad = round_up(n, 4)
     const float *kscale[kMaxLayers];  // [n]
     const float *bias[kMaxLayers];
+    // parity taps (null without them): the quantised input and every hidden layer's int8 output
+    // are also stored, rows of tap_in_pitch / tap_pitch[l] bytes
+    int8_t *tap_in, *tap[kMaxLayers];
+    int tap_in_pitch, tap_pitch[kMaxLayers];
 };
 
 __global__ void __launch_bounds__(kMaxWidth)
@@ -54,6 +58,8 @@ mlp_fused_kernel(const MlpFusedParams p, const float *__restrict__ obs, const fl
                         << (8 * j);
         }
         act[0][r][w4] = (int32_t)word;
+        if (p.tap_in && row < B && 4 * w4 < p.tap_in_pitch)
+            *reinterpret_cast<uint32_t *>(p.tap_in + (long long)row * p.tap_in_pitch + 4 * w4) = word;
     }
     __syncthreads();
 
@@ -90,7 +96,9 @@ mlp_fused_kernel(const MlpFusedParams p, const float *__restrict__ obs, const fl
                     s_logits[r][tid] = y;
                     if (row0 + r < B) logits[(long long)(row0 + r) * N + tid] = y;
                 } else {
-                    reinterpret_cast<int8_t *>(act[cur ^ 1][r])[tid] = requant(y, p.s_out[l]);
+                    const int8_t code = requant(y, p.s_out[l]);
+                    reinterpret_cast<int8_t *>(act[cur ^ 1][r])[tid] = code;
+                    if (p.tap[l] && row0 + r < B) p.tap[l][(long long)(row0 + r) * p.tap_pitch[l] + tid] = code;
                 }
             }
         } else if (!last && tid < n_pad) {
@@ -171,7 +179,15 @@ accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, 
         prm->s_out[i] = d.s_out;
         prm->kscale[i] = p->layers[i].kscale;
         prm->bias[i] = p->layers[i].bias;
+        if ((p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) && i + 1 < n_layers) {
+            prm->tap[i] = p->bufs[p->layers[i].out_buf].ptr;
+            prm->tap_pitch[i] = p->layers[i].out_cp;
+        }
         k_in = d.out_c;
+    }
+    if (p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) {
+        prm->tap_in = p->bufs[p->layers[0].in_buf].ptr;
+        prm->tap_in_pitch = p->in_cp;
     }
     p->mlp = prm;
     Step s;

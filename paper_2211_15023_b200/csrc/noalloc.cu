@@ -109,6 +109,7 @@ extern "C" accerl_status accerl_policy_act_noalloc(accerl_policy *p, const void 
     auto buf = [&](int b) { return (int8_t *)(base + offset[b]); };
 
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    p->last_stream = st;  // accerl_policy_check waits for this step
     const int B = batch;
     int8_t *x = buf(p->layers[0].in_buf);
     if (p->in_kind == ACCERL_IN_U8_NCHW)

@@ -218,7 +218,8 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
 {
     *used = false;
     if (p->in_kind != ACCERL_IN_U8_NCHW) return ACCERL_OK;
-    const bool keep = (p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) != 0;
+    const bool keep = unfuse_for_taps(p);  // every tensor must exist in an un-ReLU'd form
+    const bool tap_fused = (p->flags & ACCERL_FLAG_TAP_FUSED) != 0;
     // ---- roles
     std::vector<Role> role(n_layers);
     int n_tc = 0;
@@ -776,6 +777,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         s.tc = (int)p->tc_steps.size() - 1;
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
         if (g.fast_div) s.kernel += "[3-step divide verified]";
+        if (g.hpool) s.kernel += "[pooled along x on the accumulators]";
         steps.push_back(s);
     }
     if (!fused_sample) {
@@ -784,6 +786,14 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         ss.kernel = p->n_actions <= 32 ? "sample_warp_kernel" : "sample_wide_kernel";
         ss.covers = "sample";
         steps.push_back(ss);
+    }
+    if (tap_fused) {
+        // tensors the fused plan stores in no un-ReLU'd form cannot be tapped
+        for (int t = 1; t <= n_layers - 1; ++t) {
+            const Forms &f = forms[t];
+            p->tap_missing[t] = !(f.plain || f.pad || f.slot) ? 1 : 0;
+        }
+        if (hpool_first) p->tap_missing[1] = 1;
     }
     p->steps = steps;
     *used = true;

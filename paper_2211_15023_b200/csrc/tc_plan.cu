@@ -429,7 +429,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         // producer is written for (4 channels, space-to-depth 4, 16-byte aligned strips) and the
         // quantiser is the fixed-point line; the parity tap of the quantised input needs the
         // separate launch.
-        const bool fuse = i == 0 && d.kind == ACCERL_CONV2D && !(p->flags & ACCERL_FLAG_KEEP_ACTIVATIONS) &&
+        const bool fuse = i == 0 && d.kind == ACCERL_CONV2D && !unfuse_for_taps(p) &&
                           p->in_c == 4 && d.stride == 4 && g.chunk_bytes == 64 && g.shifted && ts.resident_b &&
                           p->ingest_arith == 1 && p->in_w % 4 == 0 && (p->in_h * p->in_w) % 16 == 0 && n_layers > 1;
         if (fuse) {
@@ -459,6 +459,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             g.a_rows = 128;
             if (!tc_choose_pipeline(g, false)) {  // generic plan stays
                 p->tensor_s2d.assign(n_layers + 1, 1);
+                p->tap_missing.assign(n_layers + 1, 0);
                 p->tc_steps.clear();
                 return ACCERL_OK;
             }
@@ -485,6 +486,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             s.kernel += "[frames quantised inside]";
             s.covers = "ingest+layer 0";
             steps.clear();
+            p->tap_missing[0] = 1;  // no quantised input tensor exists
         }
         steps.push_back(s);
     }

@@ -25,3 +25,14 @@ def pytest_collection_modifyitems(config, items):
     for it in items:
         if "gpu" in it.keywords:
             it.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter, exitstatus, config):
+    # parity counters per workload, action mismatches next to a CDF edge included
+    try:
+        import json
+        from parity_util import SESSION_STATS
+    except Exception:
+        return
+    if SESSION_STATS:
+        terminalreporter.write_line("parity counters: " + json.dumps(SESSION_STATS, sort_keys=True))

@@ -59,5 +59,29 @@ def test_noalloc_matches_act_on_two_calls_in_a_row():
     assert "scratch" in msg and str(64 * 1024 * 1024) in msg
     assert tiny.act_noalloc_raw(None, u.data_ptr(), 4, got[0].data_ptr(), got[1].data_ptr(),
                                 got[2].data_ptr(), stream) == 1
+    big.check()
+    tiny.check()    # waits on the stream of the last noalloc step, reports the device status word
+    big.close()
+    tiny.close()
+
+
+@pytest.mark.parametrize("name,b", [("cartpole_mlp", 160), ("impala_resnet_b16384", 9)])
+def test_noalloc_other_layer_kinds(name, b):
+    """fp32 vector input, max-pool and residual layers carved from the same fixed array."""
+    import paper_2211_15023_b200 as P
+    pol = W.drawn_int8_policy(name)
+    big, tiny = P.Policy(pol, b), P.Policy(pol, 1)
+    stream = torch.cuda.current_stream().cuda_stream
+    for call in range(2):
+        obs = torch.from_numpy(W.observations(name, b, seed=90 + call)).cuda()
+        u = torch.from_numpy(W.uniforms(name, b, seed=95 + call)).cuda()
+        want = big.act(obs, u)
+        got = _outputs(b, tiny.n_actions)
+        assert tiny.act_noalloc_raw(obs.data_ptr(), u.data_ptr(), b, got[0].data_ptr(),
+                                    got[1].data_ptr(), got[2].data_ptr(), stream) == 0
+        tiny.check()
+        assert np.array_equal(got[0].cpu().numpy(), want[0].cpu().numpy())
+        assert np.array_equal(got[1].cpu().numpy(), want[1].cpu().numpy())
+        np.testing.assert_allclose(got[2].cpu().numpy(), want[2].cpu().numpy(), rtol=RTOL, atol=ATOL)
     big.close()
     tiny.close()
