@@ -236,6 +236,29 @@ accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t 
                                  size_t *workspace_bytes, int32_t *launches_per_act,
                                  char *plan_buf, size_t plan_buf_bytes);
 
+/*
+ * Micro-benchmark of the int8 tensor pipe, the denominator of the tensor-core roofline (the paper
+ * has no counterpart: it measures its Actor as a whole, Introduction, Fig. 1; this measures the
+ * unit the contraction layers run on).  Launches `ctas` CTAs (one per SM up to the SM count); in
+ * each, `issuing_warps` warps issue `mmas_per_warp` tcgen05.mma kind::i8 instructions of shape
+ * M = 128, N = n, K = 32 bytes back to back on operands that already sit in shared memory, and
+ * wait (bounded) for the pipe to drain.
+ *   device              CUDA device index
+ *   n                   16 .. 256, a multiple of 16; issuing_warps * n <= 512 (tensor-memory columns)
+ *   issuing_warps       1 .. 4
+ *   mmas_per_warp       a multiple of 4, up to 2^20
+ *   ctas                1 .. 1024
+ *   ms_out              host, receives the duration of the best of three launches (CUDA events)
+ *   cycles_per_mma_out  host, receives SM cycles per MMA and CTA: mean over CTAs of
+ *                       (cycles from first issue to drained pipe) / (issuing_warps * mmas_per_warp)
+ * int8 operations per second = ctas * issuing_warps * mmas_per_warp * 2 * 128 * n * 32 / time.
+ * Synchronous; allocates and frees a few hundred bytes of device memory; uses the default stream.
+ * Errors: INVALID_ARG, UNSUPPORTED (not sm_100), CUDA, TIMEOUT (a bounded wait gave up).
+ */
+accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t issuing_warps,
+                                 int32_t mmas_per_warp, int32_t ctas, float *ms_out,
+                                 float *cycles_per_mma_out);
+
 /* Free the handle and its device memory.  Synchronises the device.  NULL is allowed. */
 void accerl_policy_destroy(accerl_policy *p);
 

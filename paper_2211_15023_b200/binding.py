@@ -58,6 +58,8 @@ def library() -> C.CDLL:
         lib.accerl_policy_check.argtypes = [vp]
         lib.accerl_policy_info.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_size_t),
                                            C.POINTER(i32), C.c_char_p, C.c_size_t]
+        lib.accerl_tc_probe_i8.argtypes = [i32, i32, i32, i32, i32, C.POINTER(f32), C.POINTER(f32)]
+        lib.accerl_tc_probe_i8.restype = C.c_int
         lib.accerl_policy_destroy.argtypes = [vp]
         lib.accerl_policy_destroy.restype = None
         lib.accerl_last_error.restype = C.c_char_p
@@ -78,6 +80,17 @@ def _out_hw(l):
         return 1, 1
     return ((l["in_h"] + 2 * l["pad"] - l["kh"]) // l["stride"] + 1,
             (l["in_w"] + 2 * l["pad"] - l["kw"]) // l["stride"] + 1)
+
+
+def tc_probe_i8(n: int, issuing_warps: int = 1, mmas_per_warp: int = 4096, ctas: int = 148,
+                device: int = 0) -> dict:
+    """accerl_tc_probe_i8: cost of an M = 128, N = n int8 MMA; returns ms, cycles_per_mma, tops."""
+    ms, cyc = C.c_float(), C.c_float()
+    _check(library().accerl_tc_probe_i8(device, n, issuing_warps, mmas_per_warp, ctas,
+                                        C.byref(ms), C.byref(cyc)))
+    ops = ctas * issuing_warps * mmas_per_warp * 2.0 * 128 * n * 32
+    return dict(n=n, issuing_warps=issuing_warps, mmas_per_warp=mmas_per_warp, ctas=ctas,
+                ms=ms.value, cycles_per_mma=cyc.value, tops=ops / (ms.value * 1e-3) / 1e12)
 
 
 class Policy:
