@@ -69,13 +69,19 @@ enum {
                                          accerl_policy_read_activation works (parity taps) */
     ACCERL_FLAG_FORCE_GENERIC = 2,    /* use only the plain CUDA-core kernels (no tensor-core
                                          or fused plans); for cross-checking the fast paths */
-    ACCERL_FLAG_TAP_FUSED = 4         /* only with KEEP_ACTIVATIONS: keep every fusion of the plan
+    ACCERL_FLAG_TAP_FUSED = 4,        /* only with KEEP_ACTIVATIONS: keep every fusion of the plan
                                          that runs without the taps (input stage inside the first
                                          conv, pooling on accumulators, the single-launch MLP) and
                                          tap the tensors that plan still stores; a tensor it never
                                          stores reads as ACCERL_ERR_UNSUPPORTED.  Without this
                                          bit KEEP_ACTIVATIONS un-fuses those steps so that every
                                          tensor exists. */
+    ACCERL_FLAG_VALUE_HEAD = 8        /* the last layer has one column more than there are actions:
+                                         columns [0, A) are the logits, column A is the state value
+                                         V(s) (Section 2.2, Eq. KD: the compressed network carries a
+                                         value function; Section 2.3, Eq. V-trace uses it).  V is the
+                                         same single fma as a logit, takes no part in the softmax and
+                                         is returned by accerl_policy_act_ex. */
 };
 
 /*
@@ -111,7 +117,8 @@ typedef struct {
  *   in_shape   host, {C, H, W}
  *   s_input    scale of the quantised input tensor (must equal layers[0].s_in)
  *   layers     host, n_layers descriptors; layer i consumes layer i-1's output; the last layer
- *              must be an FC with ACCERL_LOGITS and out_c = number of actions (1..1024)
+ *              must be an FC with ACCERL_LOGITS and out_c = number of actions (1..1024), plus one
+ *              with ACCERL_FLAG_VALUE_HEAD
  *   max_batch  largest batch `act` will be called with (>= 1)
  *   flags      ACCERL_FLAG_* bits
  * Synchronises the device once; allocates device memory (freed by accerl_policy_destroy).
@@ -140,6 +147,87 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
 accerl_status accerl_policy_act(accerl_policy *p, const void *obs_dev, const float *uniforms_dev,
                                 int32_t batch, float *logits_dev, int32_t *actions_dev,
                                 float *logp_dev, void *cuda_stream);
+
+/*
+ * accerl_policy_act with the two further per-state outputs the rest of the framework consumes:
+ *   value_dev    device, fp32 [batch], written: V(s), the value column of the last layer (Section
+ *                2.2, Eq. KD, the term with v_smaller(s); Section 2.3, Eq. V-trace, V(x_s) "estimated
+ *                by the compressed policy network").  NULL to skip; non-NULL needs a handle created
+ *                with ACCERL_FLAG_VALUE_HEAD (INVALID_ARG otherwise).
+ *   entropy_dev  device, fp32 [batch], written: H(pi(.|s)) = -sum_a p_a log p_a of the action
+ *                distribution that was sampled from (Section 2.2, Eq. KD, the regulariser; Section
+ *                2.4, one of the Monitor's indicators).  NULL to skip.
+ * Both come out of the launch that samples; everything else is as in accerl_policy_act.
+ */
+accerl_status accerl_policy_act_ex(accerl_policy *p, const void *obs_dev, const float *uniforms_dev,
+                                   int32_t batch, float *logits_dev, int32_t *actions_dev,
+                                   float *logp_dev, float *value_dev, float *entropy_dev,
+                                   void *cuda_stream);
+
+/*
+ * The Monitor's KL indicators (Section 2.4, Eq. KL): per state
+ *   KL(pi_original || pi_smaller) = sum_a pi_original(a|x) log(pi_original(a|x) / pi_smaller(a|x))
+ * from the logits two policies produced for the same batch, and optionally its mean and maximum
+ * over the batch ("KL mean", "KL max"; the paper switches 8 -> 16 bits when KL max exceeds 14).
+ *   logits_original_dev, logits_smaller_dev   device, fp32 [batch, n_actions], read only
+ *   kl_dev            device, fp32 [batch], written
+ *   kl_mean_max_dev   device, fp32 [2], written: {mean, max}; NULL to skip the reduction
+ * Enqueues one or two kernels on `cuda_stream`, returns without synchronising, allocates nothing.
+ * The reduction is done in a fixed order (same bits on every run).  Errors: INVALID_ARG, CUDA.
+ */
+accerl_status accerl_policy_kl(const float *logits_original_dev, const float *logits_smaller_dev,
+                               int32_t batch, int32_t n_actions, float *kl_dev,
+                               float *kl_mean_max_dev, void *cuda_stream);
+
+/*
+ * One Actor step in which every state follows the smaller policy with probability alpha and the
+ * original one otherwise (Section 3.2, the linear-alpha strategy between the compressed and the
+ * original network; Section 2.4, the Monitor sets alpha): state i uses `smaller` iff
+ * select_uniforms_dev[i] < alpha.  Outputs are those of the chosen policy for that state, exactly
+ * as accerl_policy_act_ex on that policy alone would give them.
+ *   smaller, original    two different handles on the same device with the same observation shape
+ *                        and number of actions; batch <= both max_batch
+ *   select_uniforms_dev  device, fp32 [batch] in [0, 1): the selector draws (independent of
+ *                        uniforms_dev, which the sampler inverts)
+ *   alpha                in [0, 1]
+ *   use_smaller_dev      device, uint8 [batch], written: 1 where `smaller` was used; NULL to skip
+ *   value_dev            needs ACCERL_FLAG_VALUE_HEAD on both handles; NULL to skip
+ * Both networks run on the whole batch and a last kernel selects per state, so the cost is the sum
+ * of the two steps; results do not depend on which other states share the batch.  The first call
+ * allocates, in `smaller`, result buffers for max_batch states (freed with the handle).  Uses both
+ * handles' workspaces: no other call on either may overlap with it on the GPU.
+ * Errors: INVALID_ARG, BATCH_TOO_LARGE, OOM, CUDA.
+ */
+accerl_status accerl_policy_act_mixed(accerl_policy *smaller, accerl_policy *original,
+                                      const void *obs_dev, const float *uniforms_dev,
+                                      const float *select_uniforms_dev, float alpha, int32_t batch,
+                                      float *logits_dev, int32_t *actions_dev, float *logp_dev,
+                                      float *value_dev, float *entropy_dev, uint8_t *use_smaller_dev,
+                                      void *cuda_stream);
+
+/*
+ * V-trace targets of the Corrector (Section 2.3, Eq. V-trace, with the clipped importance ratios
+ * rho_t = min(rho_hat, pi_original / pi_smaller), c_i = min(c_hat, pi_original / pi_smaller); the
+ * paper sets rho_hat = c_hat = 1) for `batch` rollouts of `n_steps` steps, and the advantage of
+ * Eq. A3C-V's first line:
+ *   v_s   = V(x_s) + sum_{t=s}^{n-1} (prod_{i=s}^{t-1} g_i c_i) rho_t (r_t + g_t V(x_{t+1}) - V(x_t))
+ *   adv_s = rho_s (r_s + g_s v_{s+1} - V(x_s)),        V(x_n) = v_n = bootstrap
+ * with pi_original / pi_smaller = exp(logp_original - logp_smaller) of the action taken, i.e. of
+ * the log-probs accerl_policy_act returns for the behaviour policy and the Learner's policy gives
+ * for the same actions.  g_t = gamma, or discounts[t] when that array is given (gamma times "the
+ * episode goes on", which cuts the sums at an episode end inside a rollout).
+ *   all arrays      device, fp32, time-major [n_steps, batch]; bootstrap_dev [batch]
+ *   discounts_dev   NULL, or [n_steps, batch]
+ *   vs_dev          written; adv_dev written, NULL to skip
+ * One thread per rollout runs the backward recursion the sums telescope into, in double, and
+ * rounds the results to float.  Enqueues on `cuda_stream`, returns without synchronising,
+ * allocates nothing.  Errors: INVALID_ARG, CUDA.
+ */
+accerl_status accerl_vtrace(const float *logp_smaller_dev, const float *logp_original_dev,
+                            const float *rewards_dev, const float *values_dev,
+                            const float *bootstrap_dev, const float *discounts_dev, int32_t n_steps,
+                            int32_t batch, float gamma, float rho_hat, float c_hat, float *vs_dev,
+                            float *adv_dev, void *cuda_stream);
 
 /*
  * accerl_policy_act with a stopwatch on every kernel launch, for measuring where the Actor's

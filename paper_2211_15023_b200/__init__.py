@@ -6,5 +6,6 @@ used for device memory and streams, nothing is computed in Python, and there
 is no CPU fallback -- importing :class:`Policy` without the built library
 raises.
 """
-from .binding import (AccerlError, Policy, library, library_path, FLAG_FORCE_GENERIC,  # noqa: F401
-                      FLAG_KEEP_ACTIVATIONS, FLAG_TAP_FUSED)
+from .binding import (AccerlError, Policy, act_mixed, kl, library, library_path, tc_probe_i8,  # noqa: F401
+                      vtrace, FLAG_FORCE_GENERIC, FLAG_KEEP_ACTIVATIONS, FLAG_TAP_FUSED,
+                      FLAG_VALUE_HEAD)

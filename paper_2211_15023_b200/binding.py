@@ -12,6 +12,7 @@ _LIB = None
 FLAG_KEEP_ACTIVATIONS = 1
 FLAG_FORCE_GENERIC = 2
 FLAG_TAP_FUSED = 4
+FLAG_VALUE_HEAD = 8
 RELU_IN, RELU_OUT, LOGITS = 1, 2, 4
 _KINDS = {"conv": 0, "fc": 1, "maxpool": 2}
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "BATCH_TOO_LARGE", 4: "OOM", 5: "CUDA",
@@ -58,6 +59,12 @@ def library() -> C.CDLL:
         lib.accerl_policy_check.argtypes = [vp]
         lib.accerl_policy_info.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_size_t),
                                            C.POINTER(i32), C.c_char_p, C.c_size_t]
+        lib.accerl_policy_act_ex.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+        lib.accerl_policy_kl.argtypes = [vp, vp, i32, i32, vp, vp, vp]
+        lib.accerl_policy_act_mixed.argtypes = [vp, vp, vp, vp, vp, f32, i32, vp, vp, vp, vp, vp, vp, vp]
+        lib.accerl_vtrace.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, f32, vp, vp, vp]
+        for f in ("accerl_policy_act_ex", "accerl_policy_kl", "accerl_policy_act_mixed", "accerl_vtrace"):
+            getattr(lib, f).restype = C.c_int
         lib.accerl_tc_probe_i8.argtypes = [i32, i32, i32, i32, i32, C.POINTER(f32), C.POINTER(f32)]
         lib.accerl_tc_probe_i8.restype = C.c_int
         lib.accerl_policy_destroy.argtypes = [vp]
@@ -91,6 +98,61 @@ def tc_probe_i8(n: int, issuing_warps: int = 1, mmas_per_warp: int = 4096, ctas:
     ops = ctas * issuing_warps * mmas_per_warp * 2.0 * 128 * n * 32
     return dict(n=n, issuing_warps=issuing_warps, mmas_per_warp=mmas_per_warp, ctas=ctas,
                 ms=ms.value, cycles_per_mma=cyc.value, tops=ops / (ms.value * 1e-3) / 1e12)
+
+
+def _stream_of(t, stream):
+    import torch
+    return torch.cuda.current_stream(t.device).cuda_stream if stream is None else stream
+
+
+def kl(logits_original, logits_smaller, stream=None):
+    """accerl_policy_kl on two CUDA fp32 [B, A] tensors; returns (kl [B], mean_max [2]) tensors."""
+    import torch
+    assert logits_original.shape == logits_smaller.shape and logits_original.is_contiguous() and \
+        logits_smaller.is_contiguous() and logits_original.dtype == logits_smaller.dtype == torch.float32
+    b, a = logits_original.shape
+    out = torch.empty(b, dtype=torch.float32, device=logits_original.device)
+    stats = torch.empty(2, dtype=torch.float32, device=logits_original.device)
+    _check(library().accerl_policy_kl(logits_original.data_ptr(), logits_smaller.data_ptr(), b, a,
+                                      out.data_ptr(), stats.data_ptr(), _stream_of(out, stream)))
+    return out, stats
+
+
+def vtrace(logp_smaller, logp_original, rewards, values, bootstrap, gamma, rho_hat=1.0, c_hat=1.0,
+           discounts=None, stream=None):
+    """accerl_vtrace on CUDA fp32 time-major [n, B] tensors; returns (vs, adv) tensors [n, B]."""
+    import torch
+    n, b = logp_smaller.shape
+    for t in (logp_smaller, logp_original, rewards, values):
+        assert t.shape == (n, b) and t.is_contiguous() and t.dtype == torch.float32 and t.is_cuda
+    assert bootstrap.shape == (b,) and bootstrap.is_contiguous() and bootstrap.dtype == torch.float32
+    assert discounts is None or (discounts.shape == (n, b) and discounts.is_contiguous())
+    vs, adv = torch.empty_like(values), torch.empty_like(values)
+    _check(library().accerl_vtrace(logp_smaller.data_ptr(), logp_original.data_ptr(), rewards.data_ptr(),
+                                   values.data_ptr(), bootstrap.data_ptr(),
+                                   None if discounts is None else discounts.data_ptr(), n, b,
+                                   float(gamma), float(rho_hat), float(c_hat), vs.data_ptr(),
+                                   adv.data_ptr(), _stream_of(vs, stream)))
+    return vs, adv
+
+
+def act_mixed(smaller, original, obs, uniforms, select_uniforms, alpha, stream=None):
+    """accerl_policy_act_mixed; returns dict(logits, actions, logp, entropy, use_smaller[, value])."""
+    import torch
+    b, dev = int(obs.shape[0]), obs.device
+    out = dict(logits=torch.empty((b, smaller.n_actions), dtype=torch.float32, device=dev),
+               actions=torch.empty(b, dtype=torch.int32, device=dev),
+               logp=torch.empty(b, dtype=torch.float32, device=dev),
+               entropy=torch.empty(b, dtype=torch.float32, device=dev),
+               use_smaller=torch.empty(b, dtype=torch.uint8, device=dev))
+    if smaller.value_head and original.value_head:
+        out["value"] = torch.empty(b, dtype=torch.float32, device=dev)
+    _check(library().accerl_policy_act_mixed(
+        smaller._h, original._h, obs.data_ptr(), uniforms.data_ptr(), select_uniforms.data_ptr(),
+        float(alpha), b, out["logits"].data_ptr(), out["actions"].data_ptr(), out["logp"].data_ptr(),
+        out["value"].data_ptr() if "value" in out else None, out["entropy"].data_ptr(),
+        out["use_smaller"].data_ptr(), _stream_of(obs, stream)))
+    return out
 
 
 class Policy:
@@ -128,10 +190,13 @@ class Policy:
         self.in_shape = tuple(int(v) for v in policy["in_shape"])
         self.max_batch = int(max_batch)
         self.device = int(device)
+        if self.layers[-1].get("value"):
+            flags = int(flags) | FLAG_VALUE_HEAD
         _check(lib.accerl_policy_create(C.byref(self._h), 0 if self.in_kind == "u8" else 1, shape,
                                         float(policy["s_input"]), descs, n, self.max_batch,
                                         int(flags), self.device))
-        self.n_actions = int(self.layers[-1]["out_c"])
+        self.value_head = bool(self.layers[-1].get("value"))
+        self.n_actions = int(self.layers[-1]["out_c"]) - (1 if self.value_head else 0)
 
     # -- the hot call ---------------------------------------------------------------------
     def act(self, obs, uniforms, out=None, stream=None):
@@ -151,6 +216,23 @@ class Policy:
         _check(library().accerl_policy_act(self._h, obs.data_ptr(), uniforms.data_ptr(), b,
                                            out[0].data_ptr(), out[1].data_ptr(), out[2].data_ptr(),
                                            stream))
+        return out
+
+    def act_ex(self, obs, uniforms, stream=None) -> dict:
+        """accerl_policy_act_ex: dict(logits, actions, logp, entropy[, value]) of CUDA tensors."""
+        import torch
+        b, dev = int(obs.shape[0]), obs.device
+        out = dict(logits=torch.empty((b, self.n_actions), dtype=torch.float32, device=dev),
+                   actions=torch.empty(b, dtype=torch.int32, device=dev),
+                   logp=torch.empty(b, dtype=torch.float32, device=dev),
+                   entropy=torch.empty(b, dtype=torch.float32, device=dev))
+        if self.value_head:
+            out["value"] = torch.empty(b, dtype=torch.float32, device=dev)
+        _check(library().accerl_policy_act_ex(
+            self._h, obs.data_ptr(), uniforms.data_ptr(), b, out["logits"].data_ptr(),
+            out["actions"].data_ptr(), out["logp"].data_ptr(),
+            out["value"].data_ptr() if self.value_head else None, out["entropy"].data_ptr(),
+            _stream_of(obs, stream)))
         return out
 
     def act_timed(self, obs, uniforms, out, stream=None) -> np.ndarray:

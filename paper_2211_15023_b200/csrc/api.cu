@@ -248,9 +248,12 @@ static accerl_status check_act_args(accerl_policy *p, const void *obs_dev,
 // Enqueue the plan's launches; with `ev`, record ev[i] before launch i and ev[n] after the last.
 static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const float *uniforms_dev,
                                int B, float *logits_dev, int32_t *actions_dev, float *logp_dev,
-                               cudaStream_t st, cudaEvent_t *ev)
+                               float *value_dev, float *entropy_dev, cudaStream_t st, cudaEvent_t *ev)
 {
     p->last_stream = st;
+    // a last layer with a value column and a sampler launch of its own: the layer's floats go to
+    // the handle's scratch rows of n_out, the sampler splits them into logits and value
+    float *z_dev = p->n_out != p->n_actions ? p->z_scratch : logits_dev;
     for (size_t i = 0; i < p->steps.size(); ++i) {
         const Step &s = p->steps[i];
         if (ev) ACCERL_CUDA_TRY(cudaEventRecord(ev[i], st));
@@ -273,7 +276,7 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
                 *L, in, L->skip_buf >= 0 ? p->bufs[L->skip_buf].ptr : nullptr, o, B, st));
             break;
         case Step::FC_GENERIC:
-            ACCERL_CUDA_TRY(launch_fc_generic(*L, in, o, logits_dev, B, st));
+            ACCERL_CUDA_TRY(launch_fc_generic(*L, in, o, z_dev, B, st));
             break;
         case Step::POOL_GENERIC:
             ACCERL_CUDA_TRY(launch_maxpool_generic(*L, in, o, B, st));
@@ -289,7 +292,7 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             TcGemmParams prm = t.prm;
             prm.batch = B;
             prm.m_tiles = (int)(((long long)B * prm.rows_per_image + 127) / 128);
-            prm.logits = prm.logits_mode ? logits_dev : nullptr;
+            prm.logits = prm.logits_mode ? z_dev : nullptr;
             if (prm.fuse_ingest) {
                 if ((uintptr_t)obs_dev & 15) {
                     set_error("act: this plan reads the frames with 16-byte bulk copies; obs_dev must be 16-byte aligned");
@@ -320,15 +323,16 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             break;
         case Step::MLP_FUSED:
             ACCERL_CUDA_TRY(launch_mlp_fused(p, (const float *)obs_dev, uniforms_dev, B, logits_dev,
-                                             actions_dev, logp_dev, st));
+                                             actions_dev, logp_dev, value_dev, entropy_dev, st));
             break;
         case Step::FC_SAMPLE:
             ACCERL_CUDA_TRY(launch_fc_sample(p->fc_sample, uniforms_dev, B, logits_dev, actions_dev, logp_dev,
-                                             p->sm_count, st));
+                                             value_dev, entropy_dev, p->sm_count, st));
             break;
         case Step::SAMPLE:
-            ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev,
-                                          logp_dev, st));
+            ACCERL_CUDA_TRY(launch_sample(z_dev, p->n_out, uniforms_dev, B, p->n_actions,
+                                          z_dev != logits_dev ? logits_dev : nullptr, actions_dev,
+                                          logp_dev, value_dev, entropy_dev, st));
             break;
         }
     }
@@ -374,7 +378,8 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         set_error("create: n_layers, max_batch and s_input must be positive");
         return ACCERL_ERR_INVALID_ARG;
     }
-    if (flags & ~(uint32_t)(ACCERL_FLAG_KEEP_ACTIVATIONS | ACCERL_FLAG_FORCE_GENERIC | ACCERL_FLAG_TAP_FUSED)) {
+    if (flags & ~(uint32_t)(ACCERL_FLAG_KEEP_ACTIVATIONS | ACCERL_FLAG_FORCE_GENERIC | ACCERL_FLAG_TAP_FUSED |
+                            ACCERL_FLAG_VALUE_HEAD)) {
         set_error("create: unknown flag bits 0x%x", flags);
         return ACCERL_ERR_INVALID_ARG;
     }
@@ -394,8 +399,13 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         cur = o;
         s_run = layers[i].s_out;
     }
-    if (cur.c > 1024) {
-        set_error("create: %d actions (at most 1024 supported)", cur.c);
+    const bool value_head = (flags & ACCERL_FLAG_VALUE_HEAD) != 0;
+    if (value_head && cur.c < 2) {
+        set_error("create: ACCERL_FLAG_VALUE_HEAD needs a last layer with at least two columns (actions, then V)");
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    if (cur.c - (value_head ? 1 : 0) > 1024) {
+        set_error("create: %d actions (at most 1024 supported)", cur.c - (value_head ? 1 : 0));
         return ACCERL_ERR_UNSUPPORTED;
     }
     for (int i = 0; i < n_layers; ++i) {
@@ -430,7 +440,8 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
     p->s_input = s_input;
     p->max_batch = max_batch;
     p->flags = flags;
-    p->n_actions = cur.c;
+    p->n_out = cur.c;
+    p->n_actions = cur.c - (value_head ? 1 : 0);
 
     accerl_status st = ACCERL_OK;
     auto fail = [&](accerl_status s) {
@@ -549,6 +560,19 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
                           fit_ingest_float_line(lut.data(), p->ingest_mul, p->ingest_add, &p->ingest_fa,
                                                 &p->ingest_fc1);
     }
+    if (value_head) {
+        void *d = nullptr;
+        const size_t bytes = (size_t)max_batch * p->n_out * sizeof(float) + 256;
+        cudaError_t e = cudaMalloc(&d, bytes);
+        if (e != cudaSuccess) {
+            set_error("create: cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+            cudaGetLastError();
+            return fail(e == cudaErrorMemoryAllocation ? ACCERL_ERR_OOM : ACCERL_ERR_CUDA);
+        }
+        p->owned.push_back(d);
+        p->z_scratch = (float *)d;
+        p->workspace_bytes += bytes;
+    }
     {
         std::vector<int> zero(256, 0);  // word 0 is the status; the rest is trace space
         if ((st = upload(p, zero, &p->status_word)) != ACCERL_OK) return fail(st);
@@ -618,8 +642,29 @@ accerl_status accerl_policy_act(accerl_policy *p, const void *obs_dev, const flo
                                      logp_dev);
     if (v != ACCERL_OK) return v;
     DeviceGuard guard(p->device);
-    return run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev,
+    return run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev, nullptr, nullptr,
                      (cudaStream_t)cuda_stream, nullptr);
+}
+
+accerl_status accerl_policy_act_ex(accerl_policy *p, const void *obs_dev, const float *uniforms_dev,
+                                   int32_t batch, float *logits_dev, int32_t *actions_dev,
+                                   float *logp_dev, float *value_dev, float *entropy_dev,
+                                   void *cuda_stream)
+{
+    accerl_status v = check_act_args(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev,
+                                     logp_dev);
+    if (v != ACCERL_OK) return v;
+    if (value_dev && p->n_out == p->n_actions) {
+        set_error("act_ex: value_dev given but the handle was created without ACCERL_FLAG_VALUE_HEAD");
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    if (((uintptr_t)value_dev & 3) || ((uintptr_t)entropy_dev & 3)) {
+        set_error("act_ex: misaligned pointer (value and entropy need 4 bytes)");
+        return ACCERL_ERR_INVALID_ARG;
+    }
+    DeviceGuard guard(p->device);
+    return run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev, value_dev,
+                     entropy_dev, (cudaStream_t)cuda_stream, nullptr);
 }
 
 accerl_status accerl_policy_act_timed(accerl_policy *p, const void *obs_dev,
@@ -641,7 +686,7 @@ accerl_status accerl_policy_act_timed(accerl_policy *p, const void *obs_dev,
         p->events.push_back(ev);
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    v = run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev, st,
+    v = run_steps(p, obs_dev, uniforms_dev, batch, logits_dev, actions_dev, logp_dev, nullptr, nullptr, st,
                   p->events.data());
     if (v != ACCERL_OK) return v;
     ACCERL_CUDA_TRY(cudaStreamSynchronize(st));

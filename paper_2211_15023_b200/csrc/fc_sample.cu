@@ -21,8 +21,9 @@ constexpr int kFsWarps = 8;
 
 // One row per warp, one lane per action: the arithmetic of sample_warp_kernel for a full-warp
 // segment.  Every lane returns the drawn action and its log-prob.
+template <bool ENTROPY>
 __device__ __forceinline__ void warp_sample(float z, bool live, float uu, int A, int lane, int &a,
-                                            float &lpa)
+                                            float &lpa, float &h)
 {
     if (!live) z = -INFINITY;
     float m = z;
@@ -36,6 +37,11 @@ __device__ __forceinline__ void warp_sample(float z, bool live, float uu, int A,
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     const float lp = live ? (z - m) - log1pf(s) : 0.f;
     float cdf = live ? expf(lp) : 0.f;  // inclusive scan
+    if (ENTROPY) {  // H = -sum p log p
+        h = cdf > 0.f ? -cdf * lp : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) h += __shfl_xor_sync(0xffffffffu, h, o);
+    }
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const float v = __shfl_up_sync(0xffffffffu, cdf, o);
@@ -46,9 +52,13 @@ __device__ __forceinline__ void warp_sample(float z, bool live, float uu, int A,
     lpa = __shfl_sync(0xffffffffu, lp, a);
 }
 
+// EXTRAS: the layer may have one output column more than actions, the state value V(s) (lane A;
+// no part of the softmax), and the entropy of the action distribution may be asked for.
+template <bool EXTRAS>
 __global__ void __launch_bounds__(32 * kFsWarps)
 fc_sample_kernel(const FcSampleParams q, const float *__restrict__ u, int B,
-                 float *__restrict__ logits, int32_t *__restrict__ actions, float *__restrict__ logp)
+                 float *__restrict__ logits, int32_t *__restrict__ actions, float *__restrict__ logp,
+                 float *__restrict__ value, float *__restrict__ entropy)
 {
     extern __shared__ __align__(16) int32_t fs_smem[];
     const int K4 = q.k4, A = q.n_actions;
@@ -57,6 +67,7 @@ fc_sample_kernel(const FcSampleParams q, const float *__restrict__ u, int B,
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int32_t *x0 = s_x + warp * 2 * K4, *x1 = x0 + K4;
     const bool live = lane < A;
+    const bool has_col = EXTRAS ? lane < q.n_out : live;  // a column of the layer (action or value)
     const long long stride = (long long)gridDim.x * kFsWarps;
     long long pair = (long long)blockIdx.x * kFsWarps + warp;
     // The first rows, the weights and the scales are all fetched before anything waits: the
@@ -75,7 +86,7 @@ fc_sample_kernel(const FcSampleParams q, const float *__restrict__ u, int B,
         }
     };
     fetch(pair);
-    const float ks = live ? q.kscale[lane] : 0.f, bs = live ? q.bias[lane] : 0.f;
+    const float ks = has_col ? q.kscale[lane] : 0.f, bs = has_col ? q.bias[lane] : 0.f;
     {
         const uint4 *gw = reinterpret_cast<const uint4 *>(q.w);
         uint4 *sw = reinterpret_cast<uint4 *>(s_w);
@@ -118,17 +129,25 @@ fc_sample_kernel(const FcSampleParams q, const float *__restrict__ u, int B,
             logits[row0 * A + lane] = z0;
             if (has1) logits[row1 * A + lane] = z1;
         }
+        if (EXTRAS && value && lane == A && A < q.n_out) {
+            value[row0] = z0;
+            if (has1) value[row1] = z1;
+        }
         int a;
-        float lpa;
-        warp_sample(z0, live, u0, A, lane, a, lpa);
+        float lpa, h = 0.f;
+        if (EXTRAS && entropy) warp_sample<true>(z0, live, u0, A, lane, a, lpa, h);
+        else warp_sample<false>(z0, live, u0, A, lane, a, lpa, h);
         if (lane == 0) {
             actions[row0] = a;
             logp[row0] = lpa;
+            if (EXTRAS && entropy) entropy[row0] = h;
         }
-        warp_sample(z1, live, u1, A, lane, a, lpa);
+        if (EXTRAS && entropy) warp_sample<true>(z1, live, u1, A, lane, a, lpa, h);
+        else warp_sample<false>(z1, live, u1, A, lane, a, lpa, h);
         if (lane == 0 && has1) {
             actions[row1] = a;
             logp[row1] = lpa;
+            if (EXTRAS && entropy) entropy[row1] = h;
         }
     }
 }
@@ -167,7 +186,8 @@ accerl_status build_fc_sample(accerl_policy *p, const accerl_layer_desc &d, int 
     q.x = x;
     q.pitch = pitch;
     q.k4 = K4;
-    q.n_actions = d.out_c;
+    q.n_actions = p->n_actions;
+    q.n_out = d.out_c;
     q.w = (const int32_t *)dev;
     q.kscale = L.kscale;
     q.bias = L.bias;
@@ -179,13 +199,19 @@ accerl_status build_fc_sample(accerl_policy *p, const accerl_layer_desc &d, int 
 }
 
 cudaError_t launch_fc_sample(const FcSampleParams &q, const float *u, int B, float *logits,
-                             int32_t *actions, float *logp, int sm_count, cudaStream_t st)
+                             int32_t *actions, float *logp, float *value, float *entropy, int sm_count,
+                             cudaStream_t st)
 {
     const int per_block = 2 * kFsWarps;
     long long blocks = ((long long)B + per_block - 1) / per_block;
     if (blocks > 4LL * sm_count) blocks = 4LL * sm_count;
     const size_t smem = (size_t)q.k4 * 4 * (32 + 2 * kFsWarps);
-    fc_sample_kernel<<<(unsigned)blocks, 32 * kFsWarps, smem, st>>>(q, u, B, logits, actions, logp);
+    if (value || entropy || q.n_out != q.n_actions)
+        fc_sample_kernel<true><<<(unsigned)blocks, 32 * kFsWarps, smem, st>>>(q, u, B, logits, actions, logp,
+                                                                              value, entropy);
+    else
+        fc_sample_kernel<false><<<(unsigned)blocks, 32 * kFsWarps, smem, st>>>(q, u, B, logits, actions, logp,
+                                                                               nullptr, nullptr);
     return cudaGetLastError();
 }
 

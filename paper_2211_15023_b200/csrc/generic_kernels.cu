@@ -322,12 +322,21 @@ cudaError_t launch_maxpool_generic(const LayerPlan &L, const int8_t *in, int8_t 
 // log-softmax + inverse-CDF sampling + behaviour log-prob
 // ---------------------------------------------------------------------------------------
 
+// Optional outputs of the sampler beside action and log-prob.  `z` rows are `pitch` floats apart
+// and may hold one column more than there are actions: the state value V(s) (a policy with a value
+// head), which takes no part in the softmax.  logits_out (rows of A floats) is written when the
+// logits do not already sit where the caller wants them.
+struct SampleExtras {
+    int pitch;
+    float *logits_out, *value, *entropy;
+};
+
 // A <= 32: a row occupies a power-of-two segment of a warp, one lane per action; max, sum and
 // the running CDF are segment-wide shuffles, the bucket search is a ballot.
 template <int WIDTH>
 __global__ void sample_warp_kernel(const float *__restrict__ logits, const float *__restrict__ u,
                                    int B, int A, int32_t *__restrict__ actions,
-                                   float *__restrict__ logp)
+                                   float *__restrict__ logp, const SampleExtras x)
 {
     constexpr int ROWS_PER_WARP = 32 / WIDTH;
     const int lane = threadIdx.x & 31;
@@ -335,7 +344,9 @@ __global__ void sample_warp_kernel(const float *__restrict__ logits, const float
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long row = warp * ROWS_PER_WARP + seg;
     const bool live = row < B && sl < A;
-    float z = live ? logits[row * A + sl] : -INFINITY;
+    float z = live ? logits[row * x.pitch + sl] : -INFINITY;
+    if (live && x.logits_out) x.logits_out[row * A + sl] = z;
+    if (x.value && row < B && sl == 0) x.value[row] = logits[row * x.pitch + A];
     float m = z;
 #pragma unroll
     for (int o = WIDTH / 2; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o, WIDTH));
@@ -350,6 +361,12 @@ __global__ void sample_warp_kernel(const float *__restrict__ logits, const float
     for (int o = WIDTH / 2; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o, WIDTH);
     float lp = live ? (z - m) - log1pf(s) : 0.f;
     float p = live ? expf(lp) : 0.f;
+    if (x.entropy) {  // H = -sum p log p over the segment
+        float h = p > 0.f ? -p * lp : 0.f;
+#pragma unroll
+        for (int o = WIDTH / 2; o > 0; o >>= 1) h += __shfl_xor_sync(0xffffffffu, h, o, WIDTH);
+        if (row < B && sl == 0) x.entropy[row] = h;
+    }
     float cdf = p;  // inclusive scan within the segment
 #pragma unroll
     for (int o = 1; o < WIDTH; o <<= 1) {
@@ -370,12 +387,15 @@ __global__ void sample_warp_kernel(const float *__restrict__ logits, const float
 // any A: one warp per row, lanes stride over the actions
 __global__ void sample_wide_kernel(const float *__restrict__ logits, const float *__restrict__ u,
                                    int B, int A, int32_t *__restrict__ actions,
-                                   float *__restrict__ logp)
+                                   float *__restrict__ logp, const SampleExtras x)
 {
     const int lane = threadIdx.x & 31;
     const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (row >= B) return;
-    const float *z = logits + row * A;
+    const float *z = logits + row * x.pitch;
+    if (x.logits_out)
+        for (int i = lane; i < A; i += 32) x.logits_out[row * A + i] = z[i];
+    if (x.value && lane == 0) x.value[row] = z[A];
     float m = -INFINITY;
     for (int i = lane; i < A; i += 32) m = fmaxf(m, z[i]);
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -388,6 +408,15 @@ __global__ void sample_wide_kernel(const float *__restrict__ logits, const float
         if (i != amax) s += expf(z[i] - m);
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     const float l1p = log1pf(s), uu = u[row];
+    if (x.entropy) {
+        float h = 0.f;
+        for (int i = lane; i < A; i += 32) {
+            const float lp = (z[i] - m) - l1p, p = expf(lp);
+            if (p > 0.f) h -= p * lp;
+        }
+        for (int o = 16; o > 0; o >>= 1) h += __shfl_xor_sync(0xffffffffu, h, o);
+        if (lane == 0) x.entropy[row] = h;
+    }
     float base = 0.f;
     int a = A - 1;
     bool found = false;
@@ -412,20 +441,26 @@ __global__ void sample_wide_kernel(const float *__restrict__ logits, const float
     }
 }
 
-cudaError_t launch_sample(const float *logits, const float *u, int B, int A, int32_t *actions,
-                          float *logp, cudaStream_t st)
+// z: [B][pitch] floats (pitch = A, or A + 1 with a value column); see SampleExtras
+cudaError_t launch_sample(const float *z, int pitch, const float *u, int B, int A, float *logits_out,
+                          int32_t *actions, float *logp, float *value, float *entropy, cudaStream_t st)
 {
     const int threads = 128;
     auto blocks_for = [&](int rows_per_warp) {
         long long warps = ((long long)B + rows_per_warp - 1) / rows_per_warp;
         return (unsigned)((warps * 32 + threads - 1) / threads);
     };
-    if (A <= 2) sample_warp_kernel<2><<<blocks_for(16), threads, 0, st>>>(logits, u, B, A, actions, logp);
-    else if (A <= 4) sample_warp_kernel<4><<<blocks_for(8), threads, 0, st>>>(logits, u, B, A, actions, logp);
-    else if (A <= 8) sample_warp_kernel<8><<<blocks_for(4), threads, 0, st>>>(logits, u, B, A, actions, logp);
-    else if (A <= 16) sample_warp_kernel<16><<<blocks_for(2), threads, 0, st>>>(logits, u, B, A, actions, logp);
-    else if (A <= 32) sample_warp_kernel<32><<<blocks_for(1), threads, 0, st>>>(logits, u, B, A, actions, logp);
-    else sample_wide_kernel<<<blocks_for(1), threads, 0, st>>>(logits, u, B, A, actions, logp);
+    SampleExtras x;
+    x.pitch = pitch;
+    x.logits_out = logits_out;
+    x.value = value;
+    x.entropy = entropy;
+    if (A <= 2) sample_warp_kernel<2><<<blocks_for(16), threads, 0, st>>>(z, u, B, A, actions, logp, x);
+    else if (A <= 4) sample_warp_kernel<4><<<blocks_for(8), threads, 0, st>>>(z, u, B, A, actions, logp, x);
+    else if (A <= 8) sample_warp_kernel<8><<<blocks_for(4), threads, 0, st>>>(z, u, B, A, actions, logp, x);
+    else if (A <= 16) sample_warp_kernel<16><<<blocks_for(2), threads, 0, st>>>(z, u, B, A, actions, logp, x);
+    else if (A <= 32) sample_warp_kernel<32><<<blocks_for(1), threads, 0, st>>>(z, u, B, A, actions, logp, x);
+    else sample_wide_kernel<<<blocks_for(1), threads, 0, st>>>(z, u, B, A, actions, logp, x);
     return cudaGetLastError();
 }
 

@@ -72,7 +72,8 @@ struct MlpFusedParams;  // mlp_fused.cu
 struct FcSampleParams {
     const int8_t *x;  // [B][pitch] int8 input rows
     int pitch, k4, n_actions;
-    const int32_t *w;  // [k4][32] words, lane = action
+    int n_out;         // output columns: n_actions, or n_actions + 1 with a value head
+    const int32_t *w;  // [k4][32] words, lane = output column
     const float *kscale, *bias;
 };
 
@@ -115,6 +116,9 @@ struct accerl_policy {
     int max_batch = 0;
     uint32_t flags = 0;
     int n_actions = 0;
+    int n_out = 0;                        // columns of the last layer: n_actions (+ 1 with a value head)
+    float *z_scratch = nullptr;           // device [max_batch][n_out]: last layer's floats when the
+                                          // plan's sampler is a launch of its own and n_out != n_actions
     std::vector<accerl::LayerPlan> layers;
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
     std::vector<accerl::TcStep> tc_steps;
@@ -143,6 +147,9 @@ struct accerl_policy {
     void *st_obs = nullptr;
     float *st_u = nullptr, *st_logits = nullptr, *st_logp = nullptr;
     int32_t *st_actions = nullptr;
+    // outputs of this policy inside accerl_policy_act_mixed (allocated on its first call)
+    float *mix_logits = nullptr, *mix_logp = nullptr, *mix_value = nullptr, *mix_entropy = nullptr;
+    int32_t *mix_actions = nullptr;
 };
 
 namespace accerl {
@@ -165,8 +172,8 @@ cudaError_t launch_fc_generic(const LayerPlan &L, const int8_t *in, int8_t *out,
                               int B, cudaStream_t st);
 cudaError_t launch_maxpool_generic(const LayerPlan &L, const int8_t *in, int8_t *out, int B,
                                    cudaStream_t st);
-cudaError_t launch_sample(const float *logits, const float *u, int B, int A, int32_t *actions,
-                          float *logp, cudaStream_t st);
+cudaError_t launch_sample(const float *z, int pitch, const float *u, int B, int A, float *logits_out,
+                          int32_t *actions, float *logp, float *value, float *entropy, cudaStream_t st);
 
 // tensor-core plan (tc_plan.cu): replaces p->steps when the whole network qualifies; returns
 // ACCERL_OK with *used = false when it does not
@@ -183,12 +190,14 @@ cudaError_t launch_ingest_u8_nhwc4(const uint8_t *obs, const int8_t *lut, int8_t
 accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, int n_layers,
                              bool *used);
 cudaError_t launch_mlp_fused(const accerl_policy *p, const float *obs, const float *u, int B,
-                             float *logits, int32_t *actions, float *logp, cudaStream_t st);
+                             float *logits, int32_t *actions, float *logp, float *value, float *entropy,
+                             cudaStream_t st);
 accerl_status upload_bytes(accerl_policy *p, const void *host, size_t bytes, void **dev);
 bool fc_sample_fits(const accerl_policy *p, const accerl_layer_desc *layers, int n_layers, int i);
 accerl_status build_fc_sample(accerl_policy *p, const accerl_layer_desc &d, int layer, const int8_t *x,
                               int pitch, Step *out);
 cudaError_t launch_fc_sample(const FcSampleParams &q, const float *u, int B, float *logits,
-                             int32_t *actions, float *logp, int sm_count, cudaStream_t st);
+                             int32_t *actions, float *logp, float *value, float *entropy, int sm_count,
+                             cudaStream_t st);
 
 }  // namespace accerl

@@ -39,7 +39,7 @@ struct MlpFusedParams {
 __global__ void __launch_bounds__(kMaxWidth)
 mlp_fused_kernel(const MlpFusedParams p, const float *__restrict__ obs, const float *__restrict__ u,
                  int B, float *__restrict__ logits, int32_t *__restrict__ actions,
-                 float *__restrict__ logp)
+                 float *__restrict__ logp, float *__restrict__ value, float *__restrict__ entropy)
 {
     __shared__ __align__(16) int32_t act[2][kRows][kMaxWidth / 4];
     __shared__ float s_logits[kRows][32];
@@ -92,9 +92,12 @@ mlp_fused_kernel(const MlpFusedParams p, const float *__restrict__ obs, const fl
 #pragma unroll
             for (int r = 0; r < kRows; ++r) {
                 const float y = epilogue_float(acc[r], ks, bs, p.relu[l] != 0);
-                if (last) {
+                if (last) {  // columns [0, n_actions) are logits, a further one is the state value
                     s_logits[r][tid] = y;
-                    if (row0 + r < B) logits[(long long)(row0 + r) * N + tid] = y;
+                    if (row0 + r < B) {
+                        if (tid < p.n_actions) logits[(long long)(row0 + r) * p.n_actions + tid] = y;
+                        else if (value) value[row0 + r] = y;
+                    }
                 } else {
                     const int8_t code = requant(y, p.s_out[l]);
                     reinterpret_cast<int8_t *>(act[cur ^ 1][r])[tid] = code;
@@ -124,11 +127,12 @@ mlp_fused_kernel(const MlpFusedParams p, const float *__restrict__ obs, const fl
         for (int i = 0; i < A; ++i)
             if (i != amax) s += expf(z[i] - m);
         const float l1p = log1pf(s), uu = u[row0 + tid];
-        float cdf = 0.f, lp_a = 0.f;
+        float cdf = 0.f, lp_a = 0.f, h = 0.f;
         int a = -1;
         for (int i = 0; i < A; ++i) {
-            const float lp = (z[i] - m) - l1p;
-            cdf += expf(lp);
+            const float lp = (z[i] - m) - l1p, pi = expf(lp);
+            if (pi > 0.f) h -= pi * lp;
+            cdf += pi;
             if (a < 0 && uu < cdf) {
                 a = i;
                 lp_a = lp;
@@ -140,6 +144,7 @@ mlp_fused_kernel(const MlpFusedParams p, const float *__restrict__ obs, const fl
         }
         actions[row0 + tid] = a;
         logp[row0 + tid] = lp_a;
+        if (entropy) entropy[row0 + tid] = h;
     }
 }
 
@@ -148,7 +153,7 @@ accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, 
                              bool *used)
 {
     *used = false;
-    if (p->in_kind != ACCERL_IN_F32 || n_layers > kMaxLayers || p->n_actions > 32) return ACCERL_OK;
+    if (p->in_kind != ACCERL_IN_F32 || n_layers > kMaxLayers || p->n_out > 32) return ACCERL_OK;
     if (round_up(p->in_c, 4) > kMaxWidth) return ACCERL_OK;
     for (int i = 0; i < n_layers; ++i)
         if (layers[i].kind != ACCERL_FC || layers[i].out_c > kMaxWidth ||
@@ -201,11 +206,12 @@ accerl_status build_mlp_plan(accerl_policy *p, const accerl_layer_desc *layers, 
 }
 
 cudaError_t launch_mlp_fused(const accerl_policy *p, const float *obs, const float *u, int B,
-                             float *logits, int32_t *actions, float *logp, cudaStream_t st)
+                             float *logits, int32_t *actions, float *logp, float *value, float *entropy,
+                             cudaStream_t st)
 {
     const MlpFusedParams &prm = *p->mlp;
     mlp_fused_kernel<<<(B + kRows - 1) / kRows, kMaxWidth, 0, st>>>(prm, obs, u, B, logits, actions,
-                                                                    logp);
+                                                                    logp, value, entropy);
     return cudaGetLastError();
 }
 

@@ -92,6 +92,9 @@ extern "C" accerl_status accerl_policy_act_noalloc(accerl_policy *p, const void 
         size_t bytes = p->bufs[b].bytes_per_state * (size_t)batch;
         total += (bytes + 255) / 256 * 256;
     }
+    // a value head: the last layer's rows (logits, then V) pass through the array as well
+    const size_t z_offset = total;
+    if (p->n_out != p->n_actions) total += ((size_t)batch * p->n_out * sizeof(float) + 255) / 256 * 256;
     if (total > kScratchBytes) {
         set_error("act_noalloc: batch %d needs %zu bytes of activation workspace, the built-in "
                   "scratch holds %zu (use accerl_policy_act, or a smaller batch)",
@@ -111,6 +114,7 @@ extern "C" accerl_status accerl_policy_act_noalloc(accerl_policy *p, const void 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     p->last_stream = st;  // accerl_policy_check waits for this step
     const int B = batch;
+    float *z_dev = p->n_out != p->n_actions ? (float *)(base + z_offset) : logits_dev;
     int8_t *x = buf(p->layers[0].in_buf);
     if (p->in_kind == ACCERL_IN_U8_NCHW)
         ACCERL_CUDA_TRY(launch_ingest_u8((const uint8_t *)obs_dev, p->lut, x, B, p->in_c, p->in_h,
@@ -125,11 +129,12 @@ extern "C" accerl_status accerl_policy_act_noalloc(accerl_policy *p, const void 
             ACCERL_CUDA_TRY(launch_conv_generic(L, in, L.skip_buf >= 0 ? buf(L.skip_buf) : nullptr, o,
                                                 B, st));
         else if (L.kind == ACCERL_FC)
-            ACCERL_CUDA_TRY(launch_fc_generic(L, in, o, logits_dev, B, st));
+            ACCERL_CUDA_TRY(launch_fc_generic(L, in, o, z_dev, B, st));
         else
             ACCERL_CUDA_TRY(launch_maxpool_generic(L, in, o, B, st));
     }
-    ACCERL_CUDA_TRY(launch_sample(logits_dev, uniforms_dev, B, p->n_actions, actions_dev, logp_dev,
-                                  st));
+    ACCERL_CUDA_TRY(launch_sample(z_dev, p->n_out, uniforms_dev, B, p->n_actions,
+                                  z_dev != logits_dev ? logits_dev : nullptr, actions_dev, logp_dev,
+                                  nullptr, nullptr, st));
     return ACCERL_OK;
 }

@@ -753,7 +753,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         // and move whole 128-byte lines (the load/store path bounds them otherwise)
         g.staged = (role[i] == TCPX && g.n_tile == 128 && (g.skip || g.out2)) ? 1 : 0;
         g.logits_mode = logits ? 1 : 0;
-        g.n_actions = p->n_actions;
+        g.n_actions = p->n_out;  // columns of the fp32 rows the logits layer writes
         g.status = p->status_word;
         g.trace_slot = (int)p->tc_steps.size() % 8;
         const int b_bytes = g.kstep_list ? 32 : g.chunk_bytes;  // bytes of a weight row per chunk

@@ -416,7 +416,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         g.split_cols = g.n_tile >= 128 ? 1 : 0;  // 128 / 256 columns: 32 / 64 per warpgroup
         g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
         g.logits_mode = logits ? 1 : 0;
-        g.n_actions = p->n_actions;
+        g.n_actions = p->n_out;  // columns of the fp32 rows the logits layer writes
         g.status = p->status_word;
         g.trace_slot = (int)p->tc_steps.size();
         // resident weights when the whole matrix fits beside a useful pipeline

@@ -170,6 +170,40 @@ def fp32_parameters(name: str, seed: int | None = None) -> List[dict | None]:
     return out
 
 
+def parameters_for(layers: List[dict], seed: int) -> List[dict | None]:
+    """The draw of ``fp32_parameters`` for any list of layer shapes."""
+    rng = np.random.default_rng(seed)
+    out: List[dict | None] = []
+    for l in layers:
+        if l["kind"] == "maxpool":
+            out.append(None)
+            continue
+        fan_in = l["in_c"] * l["kh"] * l["kw"]
+        w = rng.standard_normal((l["out_c"], l["in_c"], l["kh"], l["kw"])) * math.sqrt(2.0 / fan_in)
+        b = rng.standard_normal(l["out_c"]) * 0.01
+        out.append(dict(w=w.astype(np.float32), bias=b.astype(np.float32)))
+    return out
+
+
+def rollouts(n_steps: int, batch: int, seed: int, actions: int = 18, p_done: float = 0.05,
+             gamma: float = 0.99) -> dict:
+    """Synthetic Actor rollouts for the Corrector, time-major float32 [n_steps, batch]:
+    behaviour and target log-probs of the actions taken (log of a Dirichlet-like draw, so the
+    importance ratios fall on both sides of 1), rewards in {-1, 0, 1} as clipped Atari rewards
+    are, value estimates ~ N(0, 1), a bootstrap value per rollout and per-step discounts
+    (gamma, or 0 where an episode ends)."""
+    rng = np.random.default_rng(seed)
+    shape = (n_steps, batch)
+    lo = np.log(rng.dirichlet(np.ones(actions), size=shape)[..., 0] + 1e-6)
+    ls = np.log(rng.dirichlet(np.ones(actions), size=shape)[..., 0] + 1e-6)
+    return dict(logp_smaller=ls.astype(np.float32), logp_original=lo.astype(np.float32),
+                rewards=rng.integers(-1, 2, size=shape).astype(np.float32),
+                values=rng.standard_normal(shape).astype(np.float32),
+                bootstrap=rng.standard_normal(batch).astype(np.float32),
+                discounts=np.where(rng.random(shape) < p_done, 0.0, gamma).astype(np.float32),
+                gamma=gamma)
+
+
 def observations(name: str, batch: int | None = None, seed: int | None = None) -> np.ndarray:
     """A batch of states: uint8 frames [B,4,84,84] or fp32 vectors [B,D]."""
     c = CONFIGS[name]
