@@ -336,6 +336,13 @@ accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t 
  *   issuing_warps       1 .. 4
  *   mmas_per_warp       a multiple of 4, up to 2^20
  *   ctas                1 .. 1024
+ *   layout              operand layout in shared memory: 128, 64 or 32 = K-major rows of that many
+ *                       bytes under the matching swizzle; 0 = no swizzle, 16-byte K chunks in planes
+ *                       of [row][16 bytes] (8-row groups 128 bytes apart)
+ *   a_shift_rows        0 .. 128: the A operand starts this many rows into its tile, as the
+ *                       row-shifted operand views of the convolution kernels do
+ *   commit_every        0, or a multiple of 4: a tcgen05.commit (to a barrier nobody waits on)
+ *                       after every so many MMAs, as a pipeline that hands accumulators over does
  *   ms_out              host, receives the duration of the best of three launches (CUDA events)
  *   cycles_per_mma_out  host, receives SM cycles per MMA and CTA: mean over CTAs of
  *                       (cycles from first issue to drained pipe) / (issuing_warps * mmas_per_warp)
@@ -344,7 +351,8 @@ accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t 
  * Errors: INVALID_ARG, UNSUPPORTED (not sm_100), CUDA, TIMEOUT (a bounded wait gave up).
  */
 accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t issuing_warps,
-                                 int32_t mmas_per_warp, int32_t ctas, float *ms_out,
+                                 int32_t mmas_per_warp, int32_t ctas, int32_t layout,
+                                 int32_t a_shift_rows, int32_t commit_every, float *ms_out,
                                  float *cycles_per_mma_out);
 
 /* Free the handle and its device memory.  Synchronises the device.  NULL is allowed. */

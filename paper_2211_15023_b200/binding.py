@@ -65,7 +65,7 @@ def library() -> C.CDLL:
         lib.accerl_vtrace.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, f32, vp, vp, vp]
         for f in ("accerl_policy_act_ex", "accerl_policy_kl", "accerl_policy_act_mixed", "accerl_vtrace"):
             getattr(lib, f).restype = C.c_int
-        lib.accerl_tc_probe_i8.argtypes = [i32, i32, i32, i32, i32, C.POINTER(f32), C.POINTER(f32)]
+        lib.accerl_tc_probe_i8.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32, C.POINTER(f32), C.POINTER(f32)]
         lib.accerl_tc_probe_i8.restype = C.c_int
         lib.accerl_policy_destroy.argtypes = [vp]
         lib.accerl_policy_destroy.restype = None
@@ -90,13 +90,13 @@ def _out_hw(l):
 
 
 def tc_probe_i8(n: int, issuing_warps: int = 1, mmas_per_warp: int = 4096, ctas: int = 148,
-                device: int = 0) -> dict:
+                layout: int = 128, a_shift_rows: int = 0, commit_every: int = 0, device: int = 0) -> dict:
     """accerl_tc_probe_i8: cost of an M = 128, N = n int8 MMA; returns ms, cycles_per_mma, tops."""
     ms, cyc = C.c_float(), C.c_float()
-    _check(library().accerl_tc_probe_i8(device, n, issuing_warps, mmas_per_warp, ctas,
+    _check(library().accerl_tc_probe_i8(device, n, issuing_warps, mmas_per_warp, ctas, layout, a_shift_rows, commit_every,
                                         C.byref(ms), C.byref(cyc)))
     ops = ctas * issuing_warps * mmas_per_warp * 2.0 * 128 * n * 32
-    return dict(n=n, issuing_warps=issuing_warps, mmas_per_warp=mmas_per_warp, ctas=ctas,
+    return dict(n=n, issuing_warps=issuing_warps, mmas_per_warp=mmas_per_warp, ctas=ctas, layout=layout, a_shift_rows=a_shift_rows, commit_every=commit_every,
                 ms=ms.value, cycles_per_mma=cyc.value, tops=ops / (ms.value * 1e-3) / 1e12)
 
 

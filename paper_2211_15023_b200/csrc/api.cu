@@ -303,6 +303,13 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             ACCERL_CUDA_TRY(tc_launch(t.map_a, t.map_b, prm, t.resident_b, p->sm_count, st));
             break;
         }
+        case Step::CONV1_FRAMES:
+            if ((uintptr_t)obs_dev & 15) {
+                set_error("act: obs_dev must be 16-byte aligned");
+                return ACCERL_ERR_INVALID_ARG;
+            }
+            ACCERL_CUDA_TRY(conv1_launch(p->conv1_map_b, p->conv1, B, (const uint8_t *)obs_dev, p->sm_count, st));
+            break;
         case Step::INGEST_NHWC4:
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut,
                                                    p->bufs[p->layers[0].in_buf].ptr, B, p->in_h,

@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "accerl.h"
+#include "tc_conv1.h"
 #include "tc_gemm.h"
 
 namespace accerl {
@@ -51,7 +52,7 @@ struct LayerPlan {
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
     enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED,
-                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4, FC_SAMPLE } kind;
+                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4, FC_SAMPLE, CONV1_FRAMES } kind;
     int layer = -1;
     int tc = -1;  // index into accerl_policy::tc_steps (TC_GEMM) or ::pools (POOL_DUAL)
     std::string kernel, covers;
@@ -123,6 +124,8 @@ struct accerl_policy {
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
     std::vector<accerl::TcStep> tc_steps;
     std::vector<accerl::PoolDualParams> pools;
+    accerl::Conv1Params conv1 = {};       // used by a Step::CONV1_FRAMES launch
+    alignas(64) unsigned char conv1_map_b[128] = {};
     int8_t *in_pad4 = nullptr;            // frames as [n][H+2][PW][4] with the image at (1, 4)
     int in_pad4_w = 0;
     std::vector<accerl::TapDesc> taps;    // per tensor (index t + 1); empty or null ptr = generic buffer

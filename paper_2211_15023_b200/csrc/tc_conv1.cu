@@ -1,0 +1,408 @@
+// First convolution of a frame policy with the input stage inside: uint8 NCHW frames with four
+// channels, an 8 x 8 window and stride 4 (the first layer of the paper's Atari networks, table
+// "network architecture and inference time") -> int8 activations in the next layer's layout.
+//
+// The conv is a 2 x 2 stride-1 conv on the space-to-depth(4) grid of the frame: one GEMM row per
+// grid position (R, X), R = image * Hs + Y, 64 bytes of K per tap, four taps at row offsets
+// 0, 1, Ws, Ws + 1 of ONE operand block in shared memory ("shifted rows").  What differs from the
+// general contraction kernel:
+//
+// - No quantised copy of the frame ever exists, and no raw copy in shared memory either.
+//   Converter warps read the frame words straight from global memory (one lane per grid position,
+//   sixteen 4-byte loads: 4 channels x 4 image rows), quantise four bytes at a time and write the
+//   position's 64-byte operand row.  K is ordered (channel, dy, dx) -- the order the bytes have in
+//   the frame -- and the weights are permuted to match at create, so no byte is ever transposed.
+//   The next row set's loads are in flight while the current one is converted.
+// - A tile is S whole grid rows (S * Ws <= 128 GEMM rows), so a thread of the epilogue owns the
+//   same (row, X) of every tile and decodes its output address with two multiplies.  A pipeline
+//   step is T tiles; its operand block has one grid row more than it produces (the taps reach
+//   into the next row), the only data converted twice.
+// - One warp issues every MMA, eight per tile, with descriptors computed in registers: the tensor
+//   pipe takes 40 cycles for an M = 128, N <= 32 instruction (it is bound by reading the 4 KB
+//   operand from shared memory) and one thread can issue at that rate.
+// - Scales and biases are kernel parameters: the epilogue's multiply-adds take them from the
+//   constant bank, not from shared memory.
+//
+// Roles: warp 0 issues MMAs (and owns tensor memory), warps 1..3 and kFirstExtraConv.. convert,
+// warps 4..4+kEpiWarps-1 drain accumulators (warp w reads lane quarter w % 4).  Rings: kStages
+// operand blocks (full / empty barriers), kAccSlots accumulators of 32 columns (one per tile).
+// Every wait is bounded; a wait that gives up sets the status word and all roles leave.
+#include <cuda.h>
+
+#include <algorithm>
+
+#include "epilogue.cuh"
+#include "internal.h"
+#include "tc_conv1.h"
+#include "tc_ptx.cuh"
+
+namespace accerl {
+
+namespace {
+
+constexpr int kEpiWarps = 12;                       // three warpgroups
+constexpr int kConvWarps = 11;                      // converter warps (24 warps in all: 80 registers each)
+constexpr int kFirstExtraConv = 4 + kEpiWarps;      // converters beyond warps 1..3 start here
+constexpr int kWarps = 1 + kConvWarps + kEpiWarps;  // 24
+constexpr int kThreads1 = 32 * kWarps;
+constexpr int kStages = 3;
+constexpr int kAccSlots = 16;  // x 32 columns = all 512 columns of tensor memory
+constexpr int kMaxT = 4;
+
+struct __align__(8) Bars1 {
+    uint64_t full[kStages], empty[kStages];
+    uint64_t acc_full[kAccSlots], acc_empty[kAccSlots];
+    uint64_t b_ready;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+// four frame bytes -> four codes by the fixed-point line q = min((u * mul + add) >> 24, 127)
+template <bool CLAMP>
+__device__ __forceinline__ uint32_t quantise_word_line(uint32_t w, uint32_t mul, uint32_t add)
+{
+    const uint32_t r0 = __byte_perm(w, 0, 0x4440) * mul + add, r1 = __byte_perm(w, 0, 0x4441) * mul + add;
+    const uint32_t r2 = __byte_perm(w, 0, 0x4442) * mul + add, r3 = __byte_perm(w, 0, 0x4443) * mul + add;
+    const uint32_t lo = __byte_perm(r0, r1, 0x0073), hi = __byte_perm(r2, r3, 0x0073);
+    const uint32_t codes = __byte_perm(lo, hi, 0x5410);
+    return CLAMP ? __vminu4(codes, 0x7f7f7f7fu) : codes;
+}
+
+// MODE 0: line without the min, 1: line with it, 2: the table is u >> 1
+template <int MODE>
+__device__ __forceinline__ uint32_t quantise_word(uint32_t w, uint32_t mul, uint32_t add)
+{
+    if (MODE == 2) return (w >> 1) & 0x7f7f7f7fu;
+    return quantise_word_line<MODE == 1>(w, mul, add);
+}
+
+}  // namespace
+
+template <int NCOLS, int MODE>
+__global__ void __launch_bounds__(kThreads1, 1)
+conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ Conv1Params p)
+{
+    extern __shared__ __align__(1024) uint8_t smem_raw1[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw1 + 1023) & ~(uintptr_t)1023);
+    __shared__ Bars1 bars;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int kBBytes = 4 * NCOLS * 64;  // four taps of [NCOLS][64 bytes]
+    uint8_t *b_tiles = smem;
+    uint8_t *stages = smem + ((kBBytes + 1023) & ~1023);
+    const int stage_bytes = p.stage_bytes;
+    volatile int *abort_flag = &bars.abort_flag;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&bars.full[s]), (uint32_t)p.sets_per_step);
+            mbar_init(smem_u32(&bars.empty[s]), 1);
+        }
+        for (int a = 0; a < kAccSlots; ++a) {
+            mbar_init(smem_u32(&bars.acc_full[a]), 1);
+            mbar_init(smem_u32(&bars.acc_empty[a]), 4);
+        }
+        mbar_init(smem_u32(&bars.b_ready), 1);
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars.tmem_base)), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = bars.tmem_base;
+    // the next launch may set itself up while this grid drains; it waits for this grid's
+    // completion before it reads what is written here
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    const int T = p.tiles_per_step, S = p.rows_per_tile, Ws = p.grid_w;
+    const int my_steps = (int)blockIdx.x < p.total_steps
+                             ? (p.total_steps - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const uint32_t full0 = smem_u32(&bars.full[0]), empty0 = smem_u32(&bars.empty[0]);
+    const uint32_t acc_full0 = smem_u32(&bars.acc_full[0]), acc_empty0 = smem_u32(&bars.acc_empty[0]);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
+            mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)kBBytes);
+            for (int j = 0; j < 4; ++j)
+                tma_load_2d(smem_u32(b_tiles) + j * NCOLS * 64, &map_b, 0, j * NCOLS, smem_u32(&bars.b_ready));
+        }
+        __syncwarp();
+        bool ok = mbar_wait(smem_u32(&bars.b_ready), 0, abort_flag, p.status, 2);
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NCOLS >> 3) << 17) |
+                               ((uint32_t)(128 >> 4) << 24);
+        // 64-byte swizzled K-major rows: descriptor = constant upper word | (address >> 4)
+        const uint64_t desc_hi = (uint64_t)(((uint32_t)(8 * 64) >> 4) | (1u << 14) | (4u << 29)) << 32;
+        const uint32_t lo_flags = 1u << 16;
+        const uint32_t b_lo = (smem_u32(b_tiles) >> 4) | lo_flags;
+        const uint32_t tap_lo[4] = {0u, 4u, (uint32_t)(Ws * 4), (uint32_t)(Ws * 4 + 4)};  // 64-byte rows, >> 4
+        int slot = 0;
+        uint32_t slot_phase = 0;
+        for (int k = 0; k < my_steps && ok; ++k) {
+            const int step = (int)blockIdx.x + k * (int)gridDim.x;
+            const int s = k % kStages;
+            const uint32_t par = (uint32_t)((k / kStages) & 1);
+            ok = mbar_wait(full0 + 8 * s, par, abort_flag, p.status, 8);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t st_lo = ((smem_u32(stages) + (uint32_t)(s * stage_bytes)) >> 4) | lo_flags;
+            for (int i = 0; i < T && ok; ++i) {
+                if (step * T + i >= p.total_tiles) break;
+                ok = mbar_wait(acc_empty0 + 8 * slot, slot_phase ^ 1, abort_flag, p.status, 4);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (elect_one()) {
+                    const uint32_t d = tmem_base + (uint32_t)(slot * 32);
+                    const uint32_t a_lo = st_lo + (uint32_t)(i * S * Ws * 4);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+#pragma unroll
+                        for (int ks = 0; ks < 2; ++ks)
+                            mma_i8(d, desc_hi | (a_lo + tap_lo[j] + 2 * ks),
+                                   desc_hi | (b_lo + (uint32_t)(j * NCOLS * 4) + 2 * ks), idesc,
+                                   (uint32_t)(j | ks));
+                    mma_commit(acc_full0 + 8 * slot);
+                }
+                __syncwarp();
+                if (++slot == kAccSlots) {
+                    slot = 0;
+                    slot_phase ^= 1;
+                }
+            }
+            if (ok && elect_one()) mma_commit(empty0 + 8 * s);  // the block is free when these MMAs retire
+            __syncwarp();
+        }
+    } else if (warp < 4 || warp >= kFirstExtraConv) {
+        // ------------------------------------------------------------------ converters
+        // The CTA's row sets (32 grid positions each, `sets` per step) form one stream over all of its
+        // steps; warp cw takes sets cw, cw + kConvWarps, ...  Two sets are in flight per warp: while
+        // one is quantised and written, the loads of the next two travel (a single set in flight
+        // exposes the full memory latency per set).
+        const int cw = warp < 4 ? warp - 1 : warp - kFirstExtraConv + 3;
+        const int step_rows = (T * S + 1) * Ws;            // grid positions a step's block holds
+        const int sets = (step_rows + 31) / 32;            // row sets per step
+        const int total_sets = my_steps * sets;
+        const unsigned sets_magic = (unsigned)(((1ULL << 32) + sets - 1) / sets);  // exact far beyond total_sets
+        const int W = p.in_w;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        // loads of one position's sixteen words (zeros beyond the last image or the last set)
+        auto load = [&](uint32_t (&w)[16], int g) {
+            const int k = (int)__umulhi((unsigned)g, sets_magic), pos = (g - k * sets) * 32 + lane;
+            const int step = (int)blockIdx.x + k * (int)gridDim.x;
+            const int Rl = (int)__umulhi((unsigned)pos, p.ws_magic), X = pos - Rl * Ws;
+            const long long R = (long long)step * (T * S) + Rl;
+            const bool in = g < total_sets && pos < step_rows && R < p.total_grid_rows;
+            const unsigned n = __umulhi((unsigned)R, p.hs_magic);
+            const int Y = (int)((unsigned)R - n * (unsigned)p.grid_h);
+            const uint8_t *src = p.obs + (size_t)n * 4 * p.in_plane + (size_t)(4 * Y) * W + 4 * X;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int dy = 0; dy < 4; ++dy)
+                    w[4 * c + dy] = in ? __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * p.in_plane + dy * W)) : 0u;
+        };
+        bool ok = true;
+        int cur_k = -1;
+        // quantise one set and write its operand rows; the block's barrier counts one arrival per set
+        auto store = [&](const uint32_t (&w)[16], int g) {
+            const int k = (int)__umulhi((unsigned)g, sets_magic), pos = (g - k * sets) * 32 + lane;
+            const int s = k % kStages;
+            if (k != cur_k) {
+                ok = mbar_wait(empty0 + 8 * s, (uint32_t)(((k / kStages) & 1) ^ 1), abort_flag, p.status, 1);
+                ok = __all_sync(0xffffffffu, ok);
+                cur_k = k;
+                if (!ok) return;
+            }
+            uint8_t *row = stages + (size_t)s * stage_bytes + pos * 64;
+            if (pos < step_rows) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4 *>(row + ((c ^ ((pos >> 1) & 3)) << 4)) =
+                        make_uint4(quantise_word<MODE>(w[4 * c], p.ingest_mul, p.ingest_add),
+                                   quantise_word<MODE>(w[4 * c + 1], p.ingest_mul, p.ingest_add),
+                                   quantise_word<MODE>(w[4 * c + 2], p.ingest_mul, p.ingest_add),
+                                   quantise_word<MODE>(w[4 * c + 3], p.ingest_mul, p.ingest_add));
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(full0 + 8 * s);
+        };
+        uint32_t wa[16], wb[16];
+        int g = cw;
+        load(wa, g);
+        load(wb, g + kConvWarps);
+        while (g < total_sets && ok) {
+            store(wa, g);
+            load(wa, g + 2 * kConvWarps);
+            g += kConvWarps;
+            if (g >= total_sets || !ok) break;
+            store(wb, g);
+            load(wb, g + 2 * kConvWarps);
+            g += kConvWarps;
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int ew = warp - 4, wg = ew >> 2, q = warp & 3;
+        constexpr int kGroups = kEpiWarps / 4;
+        const int r = q * 32 + lane;  // this thread's row of every tile
+        const int Rl = (int)__umulhi((unsigned)r, p.ws_magic), X = r - Rl * Ws;
+        const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
+        const bool row_ok = r < S * Ws && X < p.out_w;
+        const int x_off = (X >> sh) * p.out_pitch + (X & smask) * p.n_total;
+        const float s_out = p.s_out, inv_s_out = p.inv_s_out;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        bool ok = true;
+        int seq = 0;  // tiles of this CTA so far
+        for (int k = 0; k < my_steps && ok; ++k) {
+            const int step = (int)blockIdx.x + k * (int)gridDim.x;
+            for (int i = 0; i < T; ++i, ++seq) {
+                const int tile = step * T + i;
+                if (tile >= p.total_tiles) break;
+                if (seq % kGroups != wg) continue;
+                const int slot = seq % kAccSlots;
+                const uint32_t apar = (uint32_t)((seq / kAccSlots) & 1);
+                ok = mbar_wait(acc_full0 + 8 * slot, apar, abort_flag, p.status, 16);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(slot * 32);
+                int acc[NCOLS / 16][16];
+#pragma unroll
+                for (int h = 0; h < NCOLS / 16; ++h) tmem_ld16(taddr + 16 * h, acc[h]);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_empty0 + 8 * slot);
+                const unsigned R = (unsigned)(tile * S + Rl);
+                const unsigned n = __umulhi(R, p.hs_magic);
+                const int Y = (int)(R - n * (unsigned)p.grid_h);
+                const bool valid = row_ok && Y < p.out_h && (int)n < p.batch;
+                int8_t *dst = p.out + ((size_t)n * p.out_rows_per_image + (size_t)(Y >> sh) * p.out_grid_w) * p.out_pitch +
+                              ((Y & smask) << sh) * p.n_total + x_off;
+#pragma unroll
+                for (int h = 0; h < NCOLS / 16; ++h) {
+                    float ks[16], bs[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        ks[e] = p.ks[16 * h + e];
+                        bs[e] = p.bs[16 * h + e];
+                    }
+                    uint32_t wv[4];
+                    if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                    else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                    if (valid) *reinterpret_cast<uint4 *>(dst + 16 * h) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);  // let copies in flight land
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u)
+                     : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+
+static bool magic_exact(unsigned d, unsigned long long max_x, unsigned *magic)
+{
+    const unsigned long long m = ((1ULL << 32) + d - 1) / d;
+    if (m >= (1ULL << 32)) return false;
+    *magic = (unsigned)m;
+    const unsigned long long e = m * d - (1ULL << 32);  // umulhi(x, m) = x / d while x * e < 2^32
+    return e == 0 || max_x < (1ULL << 32) / e;
+}
+
+// Does the dedicated kernel serve this first layer?  Fills everything of `q` that does not
+// depend on the call's batch or pointers.
+bool conv1_plan(const accerl_layer_desc &d, int in_h, int in_w, long long max_batch, int n_total,
+                int ingest_mode, Conv1Params *q)
+{
+    if (d.kind != ACCERL_CONV2D || d.in_c != 4 || d.kh != 8 || d.kw != 8 || d.stride != 4 || d.pad != 0 ||
+        d.skip_from >= 0 || in_h % 4 || in_w % 4 || (n_total != 16 && n_total != 32) || d.out_c != n_total)
+        return false;
+    const int Hs = in_h / 4, Ws = in_w / 4;
+    if (Ws < 2 || Ws > 64 || Hs < 2) return false;
+    const int S = 128 / Ws;
+    if (S * Ws < 112) return false;  // too many idle rows per tile
+    const long long rows = max_batch * Hs;
+    if (rows + 64 >= (1LL << 31)) return false;
+    memset(q, 0, sizeof(*q));
+    if (!magic_exact((unsigned)Ws, (unsigned long long)(kMaxT * S + 2) * Ws + 64, &q->ws_magic)) return false;
+    if (!magic_exact((unsigned)Hs, (unsigned long long)rows + 256, &q->hs_magic)) return false;
+    q->in_w = in_w;
+    q->in_plane = in_h * in_w;
+    q->grid_h = Hs;
+    q->grid_w = Ws;
+    q->rows_per_tile = S;
+    q->n_cols = n_total;
+    q->ingest_mode = ingest_mode;
+    // positions a step's MMAs can touch: (T - 1) * S * Ws + 127 + Ws + 1, plus one for the count
+    q->stage_bytes = (((kMaxT - 1) * S * Ws + 128 + Ws + 1) * 64 + 1023) & ~1023;
+    return true;
+}
+
+size_t conv1_smem_bytes(const Conv1Params &q)
+{
+    return 1024 + (((size_t)4 * q.n_cols * 64 + 1023) & ~(size_t)1023) + (size_t)kStages * q.stage_bytes;
+}
+
+cudaError_t conv1_launch(const void *map_b, const Conv1Params &q0, int batch, const uint8_t *obs,
+                         int sm_count, cudaStream_t st)
+{
+    Conv1Params q = q0;
+    q.obs = obs;
+    q.batch = batch;
+    q.total_grid_rows = (long long)batch * q.grid_h;
+    q.total_tiles = (int)((q.total_grid_rows + q.rows_per_tile - 1) / q.rows_per_tile);
+    // tiles per step: four, fewer while that leaves SMs without work
+    int T = kMaxT;
+    while (T > 1 && (q.total_tiles + T - 1) / T < 2 * sm_count) T /= 2;
+    q.tiles_per_step = T;
+    q.total_steps = (q.total_tiles + T - 1) / T;
+    q.sets_per_step = ((T * q.rows_per_tile + 1) * q.grid_w + 31) / 32;
+    const int grid = q.total_steps < sm_count ? q.total_steps : sm_count;
+    const size_t smem = conv1_smem_bytes(q);
+    auto go = [&](auto kernel) -> cudaError_t {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid);
+        cfg.blockDim = dim3(kThreads1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_b, q);
+    };
+    cudaError_t e;
+    if (q.n_cols == 32) {
+        e = q.ingest_mode == 2 ? go(conv1_frames_kernel<32, 2>)
+            : q.ingest_mode == 1 ? go(conv1_frames_kernel<32, 1>) : go(conv1_frames_kernel<32, 0>);
+    } else {
+        e = q.ingest_mode == 2 ? go(conv1_frames_kernel<16, 2>)
+            : q.ingest_mode == 1 ? go(conv1_frames_kernel<16, 1>) : go(conv1_frames_kernel<16, 0>);
+    }
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+}  // namespace accerl

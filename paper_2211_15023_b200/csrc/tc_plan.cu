@@ -453,6 +453,59 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 if (tc_smem_bytes(f, true) <= 216 * 1024) g = f;
             }
         }
+        // The dedicated first-conv kernel (tc_conv1.cu) takes the layer when it has the Atari shape:
+        // 8 x 8 window, stride 4, 16 or 32 output channels, the verified division.
+        if (fuse && g.fast_div) {
+            Conv1Params c1;
+            const int mode = p->ingest_shift1 ? 2 : (g.ingest_clamp ? 1 : 0);
+            if (conv1_plan(d, p->in_h, p->in_w, p->max_batch, n_total, mode, &c1) &&
+                conv1_smem_bytes(c1) <= 200 * 1024) {
+                c1.ingest_mul = p->ingest_mul;
+                c1.ingest_add = p->ingest_add;
+                c1.out = g.out;
+                c1.out_h = g.out_h;
+                c1.out_w = g.out_w;
+                c1.out_s2d_log2 = g.out_s2d_log2;
+                c1.out_rows_per_image = g.out_rows_per_image;
+                c1.out_grid_w = g.out_grid_w;
+                c1.out_pitch = g.out_pitch;
+                c1.n_total = n_total;
+                c1.s_out = g.s_out;
+                c1.inv_s_out = g.inv_s_out;
+                c1.relu = g.relu_out;
+                c1.status = p->status_word;
+                for (int c = 0; c < n_total; ++c) {
+                    volatile float k = d.s_in * d.s_w[c];  // one fp32 rounding, never contracted
+                    c1.ks[c] = k;
+                    c1.bs[c] = d.bias[c];
+                }
+                // weights [tap][channel][64 bytes], K ordered (c, dy, dx) as the bytes lie in the frame
+                std::vector<int8_t> w1((size_t)4 * n_total * 64, 0);
+                for (int by = 0; by < 2; ++by)
+                    for (int bx = 0; bx < 2; ++bx)
+                        for (int oc = 0; oc < d.out_c; ++oc)
+                            for (int c = 0; c < 4; ++c)
+                                for (int dy = 0; dy < 4; ++dy)
+                                    for (int dx = 0; dx < 4; ++dx)
+                                        w1[((size_t)(by * 2 + bx) * n_total + oc) * 64 + c * 16 + dy * 4 + dx] =
+                                            d.w[((oc * 4 + c) * 8 + 4 * by + dy) * 8 + 4 * bx + dx];
+                void *w1_dev = nullptr;
+                accerl_status st1 = upload_bytes(p, w1.data(), w1.size(), &w1_dev);
+                if (st1 != ACCERL_OK) return st1;
+                st1 = tc_make_map(p->conv1_map_b, w1_dev, 4LL * n_total, 64, 64, n_total, 64);
+                if (st1 != ACCERL_OK) return st1;
+                p->conv1 = c1;
+                Step s;
+                s.kind = Step::CONV1_FRAMES;
+                s.layer = i;
+                s.kernel = "conv1_frames_kernel[3-step divide verified][frames quantised inside]";
+                s.covers = "ingest+layer 0";
+                steps.clear();
+                p->tap_missing[0] = 1;  // no quantised input tensor exists
+                steps.push_back(s);
+                continue;
+            }
+        }
         if (!g.fuse_ingest && !tc_choose_pipeline(g, ts.resident_b)) {
             ts.resident_b = false;
             g.shifted = 0;

@@ -4,7 +4,7 @@
 // denominator of the tensor-core roofline and the per-instruction costs the layer plans are built
 // around (narrow tiles pay per instruction, not per multiply-accumulate).
 //
-// One CTA per SM: a 128 x 128-byte A tile and an N x 128-byte B tile (128-byte swizzle, K-major,
+// One CTA per SM: a 256 x 128-byte A tile (the MMA reads 128 rows of it, from row a_shift_rows on) and an N x 128-byte B tile (128-byte swizzle, K-major,
 // contents arbitrary) are written once; then every issuing warp's elected lane issues
 // `mmas_per_warp` MMAs back to back, walking the four 32-byte K steps of the tiles and rotating over
 // its own accumulators in tensor memory, commits, and waits (bounded) for the pipe to drain.
@@ -19,6 +19,9 @@ constexpr int kProbeMaxWarps = 4;
 
 struct ProbeParams {
     int n, warps, mmas_per_warp, acc_per_warp;
+    int commit_every;  // 0, or: a tcgen05.commit (to a barrier nobody waits on) after every so many MMAs
+    int a_shift_rows;  // the A operand starts this many rows into its tile (a row-shifted view)
+    int layout;  // bytes of a swizzled K-major operand row (128, 64, 32), or 0: no swizzle, 16-byte K chunks in planes
     unsigned long long *cycles;  // [gridDim.x] cycles between the first issue and the drained pipe
     int *status;
 };
@@ -27,15 +30,18 @@ __global__ void __launch_bounds__(32 * kProbeMaxWarps, 1) tc_probe_kernel(const 
 {
     extern __shared__ __align__(1024) uint8_t probe_smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)probe_smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ __align__(8) uint64_t done_bar[kProbeMaxWarps];
+    __shared__ __align__(8) uint64_t done_bar[kProbeMaxWarps], side_bar[kProbeMaxWarps];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint8_t *a_tile = smem, *b_tile = smem + 128 * 128;
-    for (int i = threadIdx.x; i < (128 + p.n) * 128 / 4; i += blockDim.x)
+    uint8_t *a_tile = smem, *b_tile = smem + 256 * 128;
+    for (int i = threadIdx.x; i < (256 + p.n) * 128 / 4; i += blockDim.x)
         reinterpret_cast<uint32_t *>(smem)[i] = 0x01010101u * (uint32_t)((i * 7 + 3) & 0x7f);
     if (threadIdx.x == 0) {
-        for (int w = 0; w < kProbeMaxWarps; ++w) mbar_init(smem_u32(&done_bar[w]), 1);
+        for (int w = 0; w < kProbeMaxWarps; ++w) {
+            mbar_init(smem_u32(&done_bar[w]), 1);
+            mbar_init(smem_u32(&side_bar[w]), 1);
+        }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -52,7 +58,23 @@ __global__ void __launch_bounds__(32 * kProbeMaxWarps, 1) tc_probe_kernel(const 
     const uint32_t tmem_base = tmem_base_s;
     const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.n >> 3) << 17) |
                            ((uint32_t)(128 >> 4) << 24);
-    const uint64_t adesc = make_desc(smem_u32(a_tile), 128), bdesc = make_desc(smem_u32(b_tile), 128);
+    uint64_t adesc, bdesc;
+    int ksteps;  // 32-byte K steps one operand row (or pair of planes) offers
+    if (p.layout) {
+        adesc = make_desc(smem_u32(a_tile) + (uint32_t)(p.a_shift_rows * p.layout), p.layout);
+        bdesc = make_desc(smem_u32(b_tile), p.layout);
+        ksteps = p.layout / 32;
+    } else {
+        // planes of [row][16 bytes]: 8-row groups 128 bytes apart, K chunks one plane apart
+        auto planar = [](uint32_t addr, int rows) {
+            return (uint64_t)((addr & 0x3FFFF) >> 4) | ((uint64_t)((rows * 16) >> 4) << 16) |
+                   ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
+        };
+        adesc = planar(smem_u32(a_tile) + (uint32_t)(p.a_shift_rows * 16), 256);
+        bdesc = planar(smem_u32(b_tile), p.n);
+        ksteps = 4;
+    }
+    const uint32_t a_step = p.layout ? 2u : (uint32_t)(2 * 256 * 16 >> 4), b_step = p.layout ? 2u : (uint32_t)(2 * p.n * 16 >> 4);
     long long t0 = 0;
     bool ok = true;
     if (warp < p.warps) {
@@ -65,8 +87,12 @@ __global__ void __launch_bounds__(32 * kProbeMaxWarps, 1) tc_probe_kernel(const 
             for (int i = 0; i < p.mmas_per_warp; i += 4) {
                 const uint32_t d = acc0 + (uint32_t)(a * p.n);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) mma_i8(d, adesc + 2 * k, bdesc + 2 * k, idesc, 1u);
+                for (int k = 0; k < 4; ++k) {
+                    const uint32_t kk = (uint32_t)(k & (ksteps - 1));
+                    mma_i8(d, adesc + a_step * kk, bdesc + b_step * kk, idesc, 1u);
+                }
                 if (++a == p.acc_per_warp) a = 0;
+                if (p.commit_every && (i + 4) % p.commit_every == 0) mma_commit(smem_u32(&side_bar[warp]));
             }
             mma_commit(bar);
         }
@@ -94,7 +120,8 @@ __global__ void __launch_bounds__(32 * kProbeMaxWarps, 1) tc_probe_kernel(const 
 using namespace accerl;
 
 extern "C" accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t issuing_warps,
-                                            int32_t mmas_per_warp, int32_t ctas, float *ms_out,
+                                            int32_t mmas_per_warp, int32_t ctas, int32_t layout,
+                                            int32_t a_shift_rows, int32_t commit_every, float *ms_out,
                                             float *cycles_per_mma_out)
 {
     if (!ms_out || !cycles_per_mma_out) {
@@ -103,9 +130,10 @@ extern "C" accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t i
     }
     if (n < 16 || n > 256 || n % 16 || issuing_warps < 1 || issuing_warps > kProbeMaxWarps ||
         mmas_per_warp < 4 || mmas_per_warp > (1 << 20) || mmas_per_warp % 4 || ctas < 1 || ctas > 1024 ||
-        issuing_warps * n > 512) {
+        issuing_warps * n > 512 || (layout != 0 && layout != 32 && layout != 64 && layout != 128) ||
+        a_shift_rows < 0 || a_shift_rows > 128 || commit_every < 0 || commit_every % 4) {
         set_error("tc_probe: n in 16..256 (multiple of 16), 1..4 issuing warps with warps * n <= 512, "
-                  "mmas_per_warp a multiple of 4 up to 2^20, 1..1024 CTAs");
+                  "mmas_per_warp a multiple of 4 up to 2^20, 1..1024 CTAs, layout 0, 32, 64 or 128, a_shift_rows 0..128, commit_every a multiple of 4");
         return ACCERL_ERR_INVALID_ARG;
     }
     int ndev = 0, prev = -1;
@@ -131,6 +159,9 @@ extern "C" accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t i
     q.warps = issuing_warps;
     q.mmas_per_warp = mmas_per_warp;
     q.acc_per_warp = 512 / (issuing_warps * n);
+    q.layout = layout;
+    q.a_shift_rows = a_shift_rows;
+    q.commit_every = commit_every;
     void *dev = nullptr;
     const size_t bytes = (size_t)ctas * sizeof(unsigned long long) + 64;
     ACCERL_CUDA_TRY(cudaMalloc(&dev, bytes));
@@ -141,7 +172,7 @@ extern "C" accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t i
     ACCERL_CUDA_TRY(cudaMemset(dev, 0, bytes));
     q.cycles = (unsigned long long *)dev;
     q.status = (int *)((char *)dev + (size_t)ctas * sizeof(unsigned long long));
-    const size_t smem = 1024 + (size_t)(128 + n) * 128;
+    const size_t smem = 1024 + (size_t)(256 + n) * 128;
     ACCERL_CUDA_TRY(cudaFuncSetAttribute(tc_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaEvent_t e0, e1;
     ACCERL_CUDA_TRY(cudaEventCreate(&e0));

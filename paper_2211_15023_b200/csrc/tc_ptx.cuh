@@ -56,13 +56,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after kWaitLimitPolls polls or as soon as another role has given up.
-// The pause between polls doubles up to 256 ns: a warp that waits for a whole tile must not take
-// issue slots from the working ones, one that waits briefly still wakes up quickly.
+// Bounded wait: gives up after kSpinPolls + kWaitLimitPolls polls or as soon as another role has
+// given up.  mbarrier.try_wait itself suspends the thread for a hardware-chosen interval, so the
+// first kSpinPolls polls follow each other directly: a hand-over between two roles then costs
+// the barrier's latency, not a sleep quantum (with 32..256 ns sleeps from the first miss on, every
+// hand-over of a pipeline lost up to half a microsecond).  Only a wait that lasts longer backs off
+// with pauses that double up to 256 ns, so that it does not take issue slots from working warps.
+#ifndef ACCERL_SPIN_POLLS
+#define ACCERL_SPIN_POLLS 2048
+#endif
+constexpr int kSpinPolls = ACCERL_SPIN_POLLS;
+
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                           int *status, int code)
 {
     if (mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < kSpinPolls; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63) == 63 && *abort_flag) return false;
+    }
     unsigned ns = 32;
     for (int i = 0; i < kWaitLimitPolls; ++i) {
         __nanosleep(ns);
