@@ -17,19 +17,22 @@
 //   same (row, X) of every tile and decodes its output address with two multiplies.  A pipeline
 //   step is T tiles; its operand block has one grid row more than it produces (the taps reach
 //   into the next row), the only data converted twice.
-// - One warp issues every MMA, eight per tile, with descriptors computed in registers: the tensor
-//   pipe takes 40 cycles for an M = 128, N <= 32 instruction (it is bound by reading the 4 KB
-//   operand from shared memory) and one thread can issue at that rate.
-// - Scales and biases are kernel parameters: the epilogue's multiply-adds take them from the
-//   constant bank, not from shared memory.
+// - MMA descriptors are computed in registers, eight MMAs per tile: the tensor pipe takes 40 cycles
+//   for an M = 128, N <= 32 instruction (it is bound by reading the 4 KB operand from shared
+//   memory).
+// - Scales and biases are kernel parameters, read from the constant bank: with them in shared
+//   memory the epilogue's broadcast loads queue behind the operand reads of the MMAs (measured:
+//   113 against 94 us for the layer).
 //
-// Roles: warp 0 issues MMAs (and owns tensor memory), warps 1..3 and kFirstExtraConv.. convert,
+// Roles: warps 0..kMmaWarps1-1 issue MMAs (warp 0 owns tensor memory), the rest of warps 0..3 and
+// warps kFirstExtraConv.. convert,
 // warps 4..4+kEpiWarps-1 drain accumulators (warp w reads lane quarter w % 4).  Rings: kStages
 // operand blocks (full / empty barriers), kAccSlots accumulators of 32 columns (one per tile).
 // Every wait is bounded; a wait that gives up sets the status word and all roles leave.
 #include <cuda.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "epilogue.cuh"
 #include "internal.h"
@@ -41,9 +44,10 @@ namespace accerl {
 namespace {
 
 constexpr int kEpiWarps = 12;                       // three warpgroups
-constexpr int kConvWarps = 11;                      // converter warps (24 warps in all: 80 registers each)
-constexpr int kFirstExtraConv = 4 + kEpiWarps;      // converters beyond warps 1..3 start here
-constexpr int kWarps = 1 + kConvWarps + kEpiWarps;  // 24
+constexpr int kMmaWarps1 = 2;                       // issuing warps (tiles of a step in turn)
+constexpr int kWarps = 24;                          // 768 threads: 80 registers each
+constexpr int kConvWarps = kWarps - kEpiWarps - kMmaWarps1;  // converter warps
+constexpr int kFirstExtraConv = 4 + kEpiWarps;      // converters beyond warps kMmaWarps1..3 start here
 constexpr int kThreads1 = 32 * kWarps;
 constexpr int kStages = 3;
 constexpr int kAccSlots = 16;  // x 32 columns = all 512 columns of tensor memory
@@ -78,7 +82,9 @@ __device__ __forceinline__ uint32_t quantise_word(uint32_t w, uint32_t mul, uint
 
 }  // namespace
 
-template <int NCOLS, int MODE>
+// ATARI: the frame is 84 x 84 (a 21 x 21 grid, tiles of six grid rows); the divisions, strides and
+// load offsets are then compile-time constants, which takes a third off the converters' instructions.
+template <int NCOLS, int MODE, bool ATARI>
 __global__ void __launch_bounds__(kThreads1, 1)
 conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ Conv1Params p)
 {
@@ -95,7 +101,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&bars.full[s]), (uint32_t)p.sets_per_step);
-            mbar_init(smem_u32(&bars.empty[s]), 1);
+            mbar_init(smem_u32(&bars.empty[s]), kMmaWarps1);
         }
         for (int a = 0; a < kAccSlots; ++a) {
             mbar_init(smem_u32(&bars.acc_full[a]), 1);
@@ -120,15 +126,23 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
     // completion before it reads what is written here
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    const int T = p.tiles_per_step, S = p.rows_per_tile, Ws = p.grid_w;
+    const int T = p.tiles_per_step, S = ATARI ? 6 : p.rows_per_tile, Ws = ATARI ? 21 : p.grid_w;
+    const int Hs = ATARI ? 21 : p.grid_h;
+    // x / Ws and x / Hs for the small non-negative values that occur
+    auto div_ws = [&](unsigned x) { return ATARI ? x / 21u : __umulhi(x, p.ws_magic); };
+    auto div_hs = [&](unsigned x) { return ATARI ? x / 21u : __umulhi(x, p.hs_magic); };
     const int my_steps = (int)blockIdx.x < p.total_steps
                              ? (p.total_steps - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const uint32_t full0 = smem_u32(&bars.full[0]), empty0 = smem_u32(&bars.empty[0]);
     const uint32_t acc_full0 = smem_u32(&bars.acc_full[0]), acc_empty0 = smem_u32(&bars.acc_empty[0]);
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (elect_one()) {
+    if (warp < kMmaWarps1) {
+        // ------------------------------------------------------------------ MMA issuers
+        // (an issuing warp runs a hundred-odd instructions per tile beside the eight MMAs, and a warp
+        // that shares its scheduler with five others issues one instruction every six to eight
+        // cycles: one warp alone cannot keep the tensor pipe busy, so the tiles of a step go to
+        // kMmaWarps1 warps in turn)
+        if (warp == 0 && elect_one()) {
             mbar_expect_tx(smem_u32(&bars.b_ready), (uint32_t)kBBytes);
             for (int j = 0; j < 4; ++j)
                 tma_load_2d(smem_u32(b_tiles) + j * NCOLS * 64, &map_b, 0, j * NCOLS, smem_u32(&bars.b_ready));
@@ -142,8 +156,6 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
         const uint32_t lo_flags = 1u << 16;
         const uint32_t b_lo = (smem_u32(b_tiles) >> 4) | lo_flags;
         const uint32_t tap_lo[4] = {0u, 4u, (uint32_t)(Ws * 4), (uint32_t)(Ws * 4 + 4)};  // 64-byte rows, >> 4
-        int slot = 0;
-        uint32_t slot_phase = 0;
         for (int k = 0; k < my_steps && ok; ++k) {
             const int step = (int)blockIdx.x + k * (int)gridDim.x;
             const int s = k % kStages;
@@ -152,8 +164,10 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t st_lo = ((smem_u32(stages) + (uint32_t)(s * stage_bytes)) >> 4) | lo_flags;
-            for (int i = 0; i < T && ok; ++i) {
+            for (int i = warp; i < T && ok; i += kMmaWarps1) {
                 if (step * T + i >= p.total_tiles) break;
+                const int seq = k * T + i, slot = seq % kAccSlots;  // the CTA's tiles in order
+                const uint32_t slot_phase = (uint32_t)((seq / kAccSlots) & 1);
                 ok = mbar_wait(acc_empty0 + 8 * slot, slot_phase ^ 1, abort_flag, p.status, 4);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -170,42 +184,39 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                     mma_commit(acc_full0 + 8 * slot);
                 }
                 __syncwarp();
-                if (++slot == kAccSlots) {
-                    slot = 0;
-                    slot_phase ^= 1;
-                }
             }
             if (ok && elect_one()) mma_commit(empty0 + 8 * s);  // the block is free when these MMAs retire
             __syncwarp();
         }
     } else if (warp < 4 || warp >= kFirstExtraConv) {
+        static_assert(kMmaWarps1 <= 4 && kConvWarps >= 1, "roles");
         // ------------------------------------------------------------------ converters
         // The CTA's row sets (32 grid positions each, `sets` per step) form one stream over all of its
         // steps; warp cw takes sets cw, cw + kConvWarps, ...  Two sets are in flight per warp: while
         // one is quantised and written, the loads of the next two travel (a single set in flight
         // exposes the full memory latency per set).
-        const int cw = warp < 4 ? warp - 1 : warp - kFirstExtraConv + 3;
+        const int cw = warp < 4 ? warp - kMmaWarps1 : warp - kFirstExtraConv + (4 - kMmaWarps1);
         const int step_rows = (T * S + 1) * Ws;            // grid positions a step's block holds
         const int sets = (step_rows + 31) / 32;            // row sets per step
         const int total_sets = my_steps * sets;
         const unsigned sets_magic = (unsigned)(((1ULL << 32) + sets - 1) / sets);  // exact far beyond total_sets
-        const int W = p.in_w;
+        const int W = ATARI ? 84 : p.in_w, plane = ATARI ? 84 * 84 : p.in_plane;
         asm volatile("griddepcontrol.wait;" ::: "memory");
         // loads of one position's sixteen words (zeros beyond the last image or the last set)
         auto load = [&](uint32_t (&w)[16], int g) {
             const int k = (int)__umulhi((unsigned)g, sets_magic), pos = (g - k * sets) * 32 + lane;
             const int step = (int)blockIdx.x + k * (int)gridDim.x;
-            const int Rl = (int)__umulhi((unsigned)pos, p.ws_magic), X = pos - Rl * Ws;
+            const int Rl = (int)div_ws((unsigned)pos), X = pos - Rl * Ws;
             const long long R = (long long)step * (T * S) + Rl;
             const bool in = g < total_sets && pos < step_rows && R < p.total_grid_rows;
-            const unsigned n = __umulhi((unsigned)R, p.hs_magic);
-            const int Y = (int)((unsigned)R - n * (unsigned)p.grid_h);
-            const uint8_t *src = p.obs + (size_t)n * 4 * p.in_plane + (size_t)(4 * Y) * W + 4 * X;
+            const unsigned n = div_hs((unsigned)R);
+            const int Y = (int)((unsigned)R - n * (unsigned)Hs);
+            const uint8_t *src = p.obs + (size_t)n * 4 * plane + (size_t)(4 * Y) * W + 4 * X;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int dy = 0; dy < 4; ++dy)
-                    w[4 * c + dy] = in ? __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * p.in_plane + dy * W)) : 0u;
+                    w[4 * c + dy] = in ? __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * plane + dy * W)) : 0u;
         };
         bool ok = true;
         int cur_k = -1;
@@ -251,18 +262,17 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
         const int ew = warp - 4, wg = ew >> 2, q = warp & 3;
         constexpr int kGroups = kEpiWarps / 4;
         const int r = q * 32 + lane;  // this thread's row of every tile
-        const int Rl = (int)__umulhi((unsigned)r, p.ws_magic), X = r - Rl * Ws;
+        const int Rl = (int)div_ws((unsigned)r), X = r - Rl * Ws;
         const int sh = p.out_s2d_log2, smask = (1 << sh) - 1;
         const bool row_ok = r < S * Ws && X < p.out_w;
         const int x_off = (X >> sh) * p.out_pitch + (X & smask) * p.n_total;
         const float s_out = p.s_out, inv_s_out = p.inv_s_out;
         asm volatile("griddepcontrol.wait;" ::: "memory");
         bool ok = true;
-        int seq = 0;  // tiles of this CTA so far
         for (int k = 0; k < my_steps && ok; ++k) {
             const int step = (int)blockIdx.x + k * (int)gridDim.x;
-            for (int i = 0; i < T; ++i, ++seq) {
-                const int tile = step * T + i;
+            for (int i = 0; i < T; ++i) {
+                const int tile = step * T + i, seq = k * T + i;  // seq: the CTA's tiles in order
                 if (tile >= p.total_tiles) break;
                 if (seq % kGroups != wg) continue;
                 const int slot = seq % kAccSlots;
@@ -280,8 +290,8 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_empty0 + 8 * slot);
                 const unsigned R = (unsigned)(tile * S + Rl);
-                const unsigned n = __umulhi(R, p.hs_magic);
-                const int Y = (int)(R - n * (unsigned)p.grid_h);
+                const unsigned n = div_hs(R);
+                const int Y = (int)(R - n * (unsigned)Hs);
                 const bool valid = row_ok && Y < p.out_h && (int)n < p.batch;
                 int8_t *dst = p.out + ((size_t)n * p.out_rows_per_image + (size_t)(Y >> sh) * p.out_grid_w) * p.out_pitch +
                               ((Y & smask) << sh) * p.n_total + x_off;
@@ -289,7 +299,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 for (int h = 0; h < NCOLS / 16; ++h) {
                     float ks[16], bs[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {
+                    for (int e = 0; e < 16; ++e) {  // kernel parameters: read from the constant bank
                         ks[e] = p.ks[16 * h + e];
                         bs[e] = p.bs[16 * h + e];
                     }
@@ -393,14 +403,18 @@ cudaError_t conv1_launch(const void *map_b, const Conv1Params &q0, int batch, co
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_b, q);
     };
+    const bool atari = q.in_w == 84 && q.in_plane == 84 * 84;
+    auto pick = [&](auto ncols, auto is_atari) -> cudaError_t {
+        constexpr int N = decltype(ncols)::value;
+        constexpr bool A = decltype(is_atari)::value;
+        return q.ingest_mode == 2 ? go(conv1_frames_kernel<N, 2, A>)
+               : q.ingest_mode == 1 ? go(conv1_frames_kernel<N, 1, A>) : go(conv1_frames_kernel<N, 0, A>);
+    };
     cudaError_t e;
-    if (q.n_cols == 32) {
-        e = q.ingest_mode == 2 ? go(conv1_frames_kernel<32, 2>)
-            : q.ingest_mode == 1 ? go(conv1_frames_kernel<32, 1>) : go(conv1_frames_kernel<32, 0>);
-    } else {
-        e = q.ingest_mode == 2 ? go(conv1_frames_kernel<16, 2>)
-            : q.ingest_mode == 1 ? go(conv1_frames_kernel<16, 1>) : go(conv1_frames_kernel<16, 0>);
-    }
+    if (q.n_cols == 32)
+        e = atari ? pick(std::integral_constant<int, 32>(), std::true_type()) : pick(std::integral_constant<int, 32>(), std::false_type());
+    else
+        e = atari ? pick(std::integral_constant<int, 16>(), std::true_type()) : pick(std::integral_constant<int, 16>(), std::false_type());
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

@@ -19,6 +19,7 @@ constexpr int kProbeMaxWarps = 4;
 
 struct ProbeParams {
     int n, warps, mmas_per_warp, acc_per_warp;
+    int overwrite;     // 1: the first MMA of every four overwrites its accumulator instead of adding to it
     int commit_every;  // 0, or: a tcgen05.commit (to a barrier nobody waits on) after every so many MMAs
     int a_shift_rows;  // the A operand starts this many rows into its tile (a row-shifted view)
     int layout;  // bytes of a swizzled K-major operand row (128, 64, 32), or 0: no swizzle, 16-byte K chunks in planes
@@ -83,16 +84,19 @@ __global__ void __launch_bounds__(32 * kProbeMaxWarps, 1) tc_probe_kernel(const 
         __syncwarp();
         t0 = clock64();
         if (elect_one()) {
-            int a = 0;
+            int a = 0, until_commit = p.commit_every;
             for (int i = 0; i < p.mmas_per_warp; i += 4) {
                 const uint32_t d = acc0 + (uint32_t)(a * p.n);
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     const uint32_t kk = (uint32_t)(k & (ksteps - 1));
-                    mma_i8(d, adesc + a_step * kk, bdesc + b_step * kk, idesc, 1u);
+                    mma_i8(d, adesc + a_step * kk, bdesc + b_step * kk, idesc, p.overwrite ? (uint32_t)k : 1u);
                 }
                 if (++a == p.acc_per_warp) a = 0;
-                if (p.commit_every && (i + 4) % p.commit_every == 0) mma_commit(smem_u32(&side_bar[warp]));
+                if (p.commit_every && (until_commit -= 4) <= 0) {
+                    mma_commit(smem_u32(&side_bar[warp]));
+                    until_commit = p.commit_every;
+                }
             }
             mma_commit(bar);
         }
@@ -131,7 +135,7 @@ extern "C" accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t i
     if (n < 16 || n > 256 || n % 16 || issuing_warps < 1 || issuing_warps > kProbeMaxWarps ||
         mmas_per_warp < 4 || mmas_per_warp > (1 << 20) || mmas_per_warp % 4 || ctas < 1 || ctas > 1024 ||
         issuing_warps * n > 512 || (layout != 0 && layout != 32 && layout != 64 && layout != 128) ||
-        a_shift_rows < 0 || a_shift_rows > 128 || commit_every < 0 || commit_every % 4) {
+        a_shift_rows < 0 || a_shift_rows > 128 || commit_every < 0 || (commit_every & 0xffff) % 4) {
         set_error("tc_probe: n in 16..256 (multiple of 16), 1..4 issuing warps with warps * n <= 512, "
                   "mmas_per_warp a multiple of 4 up to 2^20, 1..1024 CTAs, layout 0, 32, 64 or 128, a_shift_rows 0..128, commit_every a multiple of 4");
         return ACCERL_ERR_INVALID_ARG;
@@ -161,7 +165,8 @@ extern "C" accerl_status accerl_tc_probe_i8(int32_t device, int32_t n, int32_t i
     q.acc_per_warp = 512 / (issuing_warps * n);
     q.layout = layout;
     q.a_shift_rows = a_shift_rows;
-    q.commit_every = commit_every;
+    q.commit_every = commit_every & 0xffff;
+    q.overwrite = commit_every >> 16;
     void *dev = nullptr;
     const size_t bytes = (size_t)ctas * sizeof(unsigned long long) + 64;
     ACCERL_CUDA_TRY(cudaMalloc(&dev, bytes));

@@ -304,6 +304,42 @@ def test_input_stage_inside_first_conv_small_and_ragged_batches(name):
     g.close()
 
 
+@pytest.mark.parametrize("hw,c1,peak", [((68, 100), 16, 255), ((96, 64), 32, 200), ((84, 84), 32, 140),
+                                        ((44, 124), 16, 255)],
+                         ids=["68x100_c16_shift", "96x64_c32_line", "84x84_c32_line_clamped", "44x124_c16"])
+def test_first_conv_kernel_other_frames_and_input_tables(hw, c1, peak):
+    """The first-conv kernel with the input stage inside on frames other than 84 x 84 (grid widths
+    that leave idle rows in a tile, a grid height that is no multiple of the rows of a tile) and
+    with input tables other than u >> 1: calibration frames whose largest byte is `peak` give
+    s_input = peak / 255 / 127, a general line, with the clamp at 127 live when test frames
+    exceed the calibrated range.  Production plan with and without taps, and the un-fused plan."""
+    import paper_2211_15023_b200 as P
+    H, Wd = hw
+    rng = np.random.default_rng(H * 1000 + Wd + c1)
+    h1, w1 = (H - 8) // 4 + 1, (Wd - 8) // 4 + 1
+    h2, w2 = (h1 - 4) // 2 + 1, (w1 - 4) // 2 + 1
+    layers = [W._conv(4, H, Wd, c1, 8, 4, 0), W._conv(c1, h1, w1, 16, 4, 2, 0) if h1 % 2 == 0 and w1 % 2 == 0
+              else W._conv(c1, h1, w1, 16, 3, 1, 0)]
+    if layers[1]["kh"] == 3:
+        h2, w2 = h1 - 2, w1 - 2
+    layers += [W._fc(16 * h2 * w2, 64), W._fc(64, 5, relu_out=False, logits=True)]
+    params = W.parameters_for(layers, 11)
+    calib = rng.integers(0, peak + 1, (16, 4, H, Wd), dtype=np.uint8)
+    pol = oracle.calibrate("u8", (4, H, Wd), layers, params, calib)
+    b = 23
+    obs = rng.integers(0, 256, (b, 4, H, Wd), dtype=np.uint8)
+    u = rng.random(b, dtype=np.float32)
+    ref = oracle.forward(pol, obs, u)
+    for flags in (0, 5, 1):
+        g = P.Policy(pol, b, flags=flags)
+        plan = g.info()["plan"]
+        assert ("conv1_frames_kernel" in plan) == (flags != 1), plan
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        g.check()
+        compare(ref, *out, taps=g.read_activation if flags else None)
+        g.close()
+
+
 def test_exact_ties_on_the_tensor_core_path():
     """Power-of-two scales make many epilogue quotients land exactly on k + 0.5: the requantiser
     must round them to even exactly as the IEEE divide + rintf of the definition does."""
