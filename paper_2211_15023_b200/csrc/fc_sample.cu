@@ -85,13 +85,18 @@ fc_sample_kernel(const FcSampleParams q, const float *__restrict__ u, int B,
             r1[j] = (in && row1 < B) ? __ldg(g1 + i) : make_uint4(0, 0, 0, 0);
         }
     };
-    fetch(pair);
+    // Programmatic dependent launch: the weights and scales do not depend on the previous launch,
+    // so they are fetched while it drains; the rows it wrote are read after the wait.  (No early
+    // trigger of its own: a next step's first layer that starts while this kernel still runs takes
+    // its SMs' issue slots just to wait -- measured 194 against 177 us per Nature-CNN step.)
     const float ks = has_col ? q.kscale[lane] : 0.f, bs = has_col ? q.bias[lane] : 0.f;
     {
         const uint4 *gw = reinterpret_cast<const uint4 *>(q.w);
         uint4 *sw = reinterpret_cast<uint4 *>(s_w);
         for (int i = threadIdx.x; i < K4 * 8; i += blockDim.x) sw[i] = __ldg(gw + i);
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    fetch(pair);
     __syncthreads();
     for (; 2 * pair < B; pair += stride) {
         const long long row0 = 2 * pair, row1 = row0 + 1;
@@ -206,12 +211,21 @@ cudaError_t launch_fc_sample(const FcSampleParams &q, const float *u, int B, flo
     long long blocks = ((long long)B + per_block - 1) / per_block;
     if (blocks > 4LL * sm_count) blocks = 4LL * sm_count;
     const size_t smem = (size_t)q.k4 * 4 * (32 + 2 * kFsWarps);
-    if (value || entropy || q.n_out != q.n_actions)
-        fc_sample_kernel<true><<<(unsigned)blocks, 32 * kFsWarps, smem, st>>>(q, u, B, logits, actions, logp,
-                                                                              value, entropy);
-    else
-        fc_sample_kernel<false><<<(unsigned)blocks, 32 * kFsWarps, smem, st>>>(q, u, B, logits, actions, logp,
-                                                                               nullptr, nullptr);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(32 * kFsWarps);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const bool extras = value || entropy || q.n_out != q.n_actions;
+    cudaError_t e = extras ? cudaLaunchKernelEx(&cfg, fc_sample_kernel<true>, q, u, B, logits, actions, logp, value, entropy)
+                           : cudaLaunchKernelEx(&cfg, fc_sample_kernel<false>, q, u, B, logits, actions, logp,
+                                                (float *)nullptr, (float *)nullptr);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
