@@ -96,6 +96,87 @@ class ClockSampler:
                     samples=len(sm))
 
 
+# plain-ALU issue peak: SMs x 4 schedulers x 32 lanes x SM clock (lane-instructions per second)
+def alu_peak(sm_count: int, sm_mhz: float) -> float:
+    return sm_count * 4 * 32 * sm_mhz * 1e6
+
+
+def int8_probe(P) -> dict:
+    """Measured cost of the int8 tensor-core instruction (M = 128, K = 32 bytes) by width N, with
+    operands resident in shared memory: cycles per MMA and CTA, and chip-wide TOP/s.  The N = 256
+    figure is the measured dense int8 peak the tensor roofline is taken against."""
+    out = {}
+    for n in (16, 32, 64, 128, 256):
+        warps = 2 if n == 256 else 4
+        r = P.tc_probe_i8(n, warps, 4096, 148)
+        out["n%d" % n] = dict(cycles_per_mma=round(r["cycles_per_mma"], 2), tops=round(r["tops"], 1))
+    return out
+
+
+def latency_profile(P, torch, name: str, device: int, calls: int = 60) -> dict:
+    """Latency of single act calls at the workload's batch: CUDA events around every call, one call
+    at a time.  warm: the same input buffer every call; cold: a buffer larger than L2 is written
+    between calls (outside the timed events), so inputs, weights and workspace come from HBM."""
+    batch = W.config(name)["batch"]
+    g = P.Policy(W.drawn_int8_policy(name), batch, device=device)
+    dev = "cuda:%d" % device
+    obs = torch.from_numpy(W.observations(name, batch)).to(dev)
+    u = torch.from_numpy(W.uniforms(name, batch)).to(dev)
+    out = g.act(obs, u)
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(obs.device)
+    res = {}
+    for mode in ("warm", "cold"):
+        for _ in range(10):
+            g.act(obs, u, out, stream.cuda_stream)
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(calls):
+            if mode == "cold":
+                flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            g.act(obs, u, out, stream.cuda_stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        ts = np.sort(np.array(ts))
+        res[mode] = dict(p10_us=float(np.percentile(ts, 10)), p50_us=float(np.percentile(ts, 50)),
+                         p90_us=float(np.percentile(ts, 90)))
+    g.check()
+    g.close()
+    res["calls"] = calls
+    res["batch"] = batch
+    return res
+
+
+def vtrace_line(P, torch, pk: dict, device: int, n_steps: int = 16, batch: int = 8192) -> dict:
+    """The V-trace kernel on [n_steps, batch] rollouts: 4 input + 2 output floats per element."""
+    dev = "cuda:%d" % device
+    r = W.rollouts(n_steps, batch, seed=1)
+    t = {k: torch.from_numpy(r[k]).to(dev) for k in ("logp_smaller", "logp_original", "rewards", "values",
+                                                      "bootstrap")}
+    args = (t["logp_smaller"], t["logp_original"], t["rewards"], t["values"], t["bootstrap"], r["gamma"])
+    out = (torch.empty_like(t["values"]), torch.empty_like(t["values"]))
+    stream = torch.cuda.current_stream(out[0].device).cuda_stream
+    for _ in range(5):
+        P.vtrace(*args, stream=stream, out=out, checked=False)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 200
+    e0.record()
+    for _ in range(reps):
+        P.vtrace(*args, stream=stream, out=out, checked=False)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1e3
+    nbytes = 4 * (6 * n_steps * batch + batch)
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return dict(n_steps=n_steps, batch=batch, us_per_call=us, bytes=nbytes, achieved_gbs=gbs,
+                frac_of_hbm=gbs / pk["hbm_gbs"],
+                note="launch-latency bound at this size: %.1f MB per call" % (nbytes / 1e6))
+
+
 def algorithmic(name: str, batch: int) -> dict:
     """Algorithmic work of one step: 2 x useful MACs, and input + output bytes per state.
 
@@ -110,11 +191,9 @@ def algorithmic(name: str, batch: int) -> dict:
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch / states of that launch, from
 # profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 173.52 MB read + 48.61 MB written by the
 # first conv with the input stage inside)
-NCU_DRAM_BYTES_PER_STATE = {
-    ("nature_cnn_b8192",
-     "tc_gemm_kernel<resident weights>[3-step divide verified][frames quantised inside]"):
-        (173518848 + 48606464) / 6144,
-}
+NCU_DRAM_BYTES_PER_STATE = {}
+# warp-level instructions executed per state by the dominant kernel, from the same capture
+NCU_WARP_INST_PER_STATE = {}
 
 
 def launch_work(name: str, plan: str, batch: int) -> list:
@@ -131,6 +210,8 @@ def launch_work(name: str, plan: str, batch: int) -> list:
 
     out = []
     for line in plan.strip().splitlines():
+        if not line.startswith("launch "):
+            continue
         head, rest = line.split(" covers ", 1)
         kernel = head.split(": ", 1)[1]
         covers = rest.split(" (")[0]
@@ -336,7 +417,11 @@ def main() -> None:
     work = launch_work(name, r["info"]["plan"], batch)
     per = r["per_launch_ms"]
     top = int(np.argmax(per))
-    int8_peak = 2.0 * pk["bf16_tflops"]  # dense int8 = 2 x dense bf16 (nominal ratio) x measured
+    # dense int8 peak: measured by the library's probe (N = 256 MMAs back to back, operands resident
+    # in shared memory, all SMs); the nominal figure 2 x measured bf16 burst is reported beside it
+    probe = int8_probe(P)
+    int8_peak_nominal = 2.0 * pk["bf16_tflops"]
+    int8_peak = probe["n256"]["tops"]
     t_tensor = work[top]["ops"] / (int8_peak * 1e12)
     t_hbm = work[top]["bytes"] / (pk["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm:
@@ -353,10 +438,21 @@ def main() -> None:
     traffic = None if per_state is None else per_state * batch
     roof.update(traffic=traffic, kernel=work[top]["kernel"], covers=work[top]["covers"],
                 kernel_ms=float(per[top]), share=float(per[top] / per.sum()),
-                peak_source="%s (int8 = 2 x bf16 burst)" % pk["source"] if roof["bound"] == "tensor"
+                peak_source="measured int8 probe (tcgen05.mma kind::i8, M=128 N=256)" if roof["bound"] == "tensor"
                 else pk["source"])
+    # third bound: plain instruction issue (warp instructions of the committed ncu capture x 32 lanes)
+    wi = NCU_WARP_INST_PER_STATE.get((name, work[top]["kernel"]))
+    sm_mhz = (clocks or {}).get("sm_mhz") or 1965.0
+    if wi is not None:
+        lane_rate = wi * 32 * batch / (per[top] * 1e-3)
+        roof["alu"] = dict(warp_inst_per_state=wi, achieved_lane_inst_per_s=lane_rate,
+                           peak=alu_peak(148, sm_mhz), frac=lane_rate / alu_peak(148, sm_mhz),
+                           note="148 SMs x 4 schedulers x 32 lanes x SM clock")
     whole = algorithmic(name, batch)
-    step_floor_ms = max(whole["ops"] / (int8_peak * 1e12), whole["bytes"] / (pk["hbm_gbs"] * 1e9)) * 1e3
+    t_floor_tensor = whole["ops"] / (int8_peak * 1e12) * 1e3
+    t_floor_hbm = whole["bytes"] / (pk["hbm_gbs"] * 1e9) * 1e3
+    step_floor_ms = max(t_floor_tensor, t_floor_hbm)
+    step_floor_nominal_ms = max(whole["ops"] / (int8_peak_nominal * 1e12) * 1e3, t_floor_hbm)
     launches = [dict(kernel=w["kernel"], covers=w["covers"], ms=float(m)) for w, m in zip(work, per)]
 
     # ---- the other workloads, briefly (kernel-resident timing only)
@@ -372,12 +468,18 @@ def main() -> None:
             o = time_workload(P, torch, other, ob, max(5, args.steps // 2), 3, nb, local)
             w = algorithmic(other, ob)
             floor = max(w["ops"] / (int8_peak * 1e12), w["bytes"] / (pk["hbm_gbs"] * 1e9)) * 1e3
+            floor_nom = max(w["ops"] / (int8_peak_nominal * 1e12), w["bytes"] / (pk["hbm_gbs"] * 1e9)) * 1e3
             others[other] = dict(batch=ob, ms_per_step=o["ms"], states_per_s=ob / (o["ms"] * 1e-3),
                                  launches=o["info"]["launches_per_act"],
                                  ops_per_state=w["ops"] // ob,
                                  ops_per_state_dense_executed=w["ops_dense_executed"] // ob,
-                                 frac_of_step_roofline=floor / o["ms"])
+                                 frac_of_step_roofline=floor / o["ms"],
+                                 frac_of_step_roofline_nominal_int8=floor_nom / o["ms"])
             o["policy"].close()
+        # latency of single calls for the small-batch configurations, and the V-trace kernel
+        for small in ("cartpole_mlp", "lunarlander_mlp", "nature_cnn_b160"):
+            others[small]["latency"] = latency_profile(P, torch, small, local)
+        others["vtrace"] = vtrace_line(P, torch, pk, local)
 
     # ---- CPU oracle on a bounded sample of the same workload (reported baseline)
     # and the parity of what was timed: the GPU outputs of those states (same policy, same plan,
@@ -394,6 +496,20 @@ def main() -> None:
         cpu_dt = time.perf_counter() - t0
         cpu = dict(value=sample / cpu_dt, unit=UNIT, cores=os.cpu_count(), kind="oracle",
                    sample="first %d states of the %d-state batch, one pass" % (sample, batch))
+        # the same oracle on one thread (a smaller sample; work per state is constant)
+        try:
+            import ctypes
+            gomp = ctypes.CDLL("libgomp.so.1")
+            n_thr = gomp.omp_get_max_threads()
+            gomp.omp_set_num_threads(1)
+            one = max(8, sample // 32)
+            t0 = time.perf_counter()
+            oracle.forward(pol, so[:one], su[:one], keep=False)
+            cpu["single_thread"] = dict(value=one / (time.perf_counter() - t0), unit=UNIT, sample="%d states" % one)
+            gomp.omp_set_num_threads(n_thr)
+            cpu["cores"] = int(n_thr)
+        except OSError:
+            pass
         lg, ac, lp = (a[:sample] for a in check_out)
         diff = ac != ref["actions"]
         same = ~diff
@@ -420,7 +536,13 @@ def main() -> None:
                 "d2h_bytes_per_step": OUT_BYTES(a) * batch},
         "gpu_launches": int(len(per) * args.steps),
         "roofline": roof,
+        "int8_probe": probe,
         "step_roofline": {"floor_ms": step_floor_ms, "frac": step_floor_ms / ms,
+                          "floor_tensor_ms": t_floor_tensor, "floor_hbm_ms": t_floor_hbm,
+                          "int8_peak_tops": int8_peak, "int8_peak_source": "measured probe, N=256",
+                          "floor_ms_nominal_int8": step_floor_nominal_ms,
+                          "frac_nominal_int8": step_floor_nominal_ms / ms,
+                          "int8_peak_nominal_tops": int8_peak_nominal,
                           "ops_per_state": whole["ops"] // batch,
                           "ops_per_state_dense_executed": whole["ops_dense_executed"] // batch,
                           "bytes_per_state": whole["bytes"] // batch},

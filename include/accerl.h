@@ -76,12 +76,19 @@ enum {
                                          stores reads as ACCERL_ERR_UNSUPPORTED.  Without this
                                          bit KEEP_ACTIVATIONS un-fuses those steps so that every
                                          tensor exists. */
-    ACCERL_FLAG_VALUE_HEAD = 8        /* the last layer has one column more than there are actions:
+    ACCERL_FLAG_VALUE_HEAD = 8,       /* the last layer has one column more than there are actions:
                                          columns [0, A) are the logits, column A is the state value
                                          V(s) (Section 2.2, Eq. KD: the compressed network carries a
                                          value function; Section 2.3, Eq. V-trace uses it).  V is the
                                          same single fma as a logit, takes no part in the softmax and
                                          is returned by accerl_policy_act_ex. */
+    ACCERL_FLAG_TEST_NO_FASTDIV = 16  /* test hook: treat every output scale as one for which the
+                                         division-free requantiser could not be verified at create.
+                                         Layers then run the epilogue that re-does elements near a
+                                         rounding tie with the IEEE divide, and plans that have no
+                                         such epilogue give way to the plain CUDA-core kernels --
+                                         what a policy with an unlucky scale gets.  Results are
+                                         the same bits either way. */
 };
 
 /*
@@ -314,9 +321,19 @@ accerl_status accerl_policy_read_activation(accerl_policy *p, int32_t layer, int
 accerl_status accerl_policy_check(accerl_policy *p);
 
 /*
+ * Exercise the give-up path of the library's bounded device-side waits (the paper has no
+ * counterpart: robustness support).  Enqueues a one-warp kernel that waits on a barrier nothing
+ * arrives at, for at most `poll_limit` polls (1 .. 100000, at most 256 ns apart); the wait runs out,
+ * the kernel sets the handle's status word and returns normally.  The next accerl_policy_check
+ * reports ACCERL_ERR_TIMEOUT and clears the word; the handle and the context stay usable.
+ */
+accerl_status accerl_policy_selftest_wait(accerl_policy *p, int32_t poll_limit, void *cuda_stream);
+
+/*
  * Describe the handle: number of actions, bytes of device workspace, kernel launches per
- * `act` call and a human-readable plan (one line per launch) written as a NUL-terminated
- * string into plan_buf (truncated to plan_buf_bytes).  Any output pointer may be NULL.
+ * `act` call and a human-readable plan (one "launch i: ..." line per launch, then a "note: ..."
+ * line if a faster plan had to be passed over and why) written as a NUL-terminated string into
+ * plan_buf (truncated to plan_buf_bytes).  Any output pointer may be NULL.
  * The plan is fixed at create time for max_batch; `batch` is accepted for symmetry with the act
  * calls and does not change the answer.
  */

@@ -13,6 +13,7 @@ FLAG_KEEP_ACTIVATIONS = 1
 FLAG_FORCE_GENERIC = 2
 FLAG_TAP_FUSED = 4
 FLAG_VALUE_HEAD = 8
+FLAG_TEST_NO_FASTDIV = 16
 RELU_IN, RELU_OUT, LOGITS = 1, 2, 4
 _KINDS = {"conv": 0, "fc": 1, "maxpool": 2}
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "BATCH_TOO_LARGE", 4: "OOM", 5: "CUDA",
@@ -65,6 +66,8 @@ def library() -> C.CDLL:
         lib.accerl_vtrace.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, f32, vp, vp, vp]
         for f in ("accerl_policy_act_ex", "accerl_policy_kl", "accerl_policy_act_mixed", "accerl_vtrace"):
             getattr(lib, f).restype = C.c_int
+        lib.accerl_policy_selftest_wait.argtypes = [vp, i32, vp]
+        lib.accerl_policy_selftest_wait.restype = C.c_int
         lib.accerl_tc_probe_i8.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32, C.POINTER(f32), C.POINTER(f32)]
         lib.accerl_tc_probe_i8.restype = C.c_int
         lib.accerl_policy_destroy.argtypes = [vp]
@@ -119,15 +122,16 @@ def kl(logits_original, logits_smaller, stream=None):
 
 
 def vtrace(logp_smaller, logp_original, rewards, values, bootstrap, gamma, rho_hat=1.0, c_hat=1.0,
-           discounts=None, stream=None):
+           discounts=None, stream=None, out=None, checked=True):
     """accerl_vtrace on CUDA fp32 time-major [n, B] tensors; returns (vs, adv) tensors [n, B]."""
     import torch
     n, b = logp_smaller.shape
-    for t in (logp_smaller, logp_original, rewards, values):
-        assert t.shape == (n, b) and t.is_contiguous() and t.dtype == torch.float32 and t.is_cuda
-    assert bootstrap.shape == (b,) and bootstrap.is_contiguous() and bootstrap.dtype == torch.float32
-    assert discounts is None or (discounts.shape == (n, b) and discounts.is_contiguous())
-    vs, adv = torch.empty_like(values), torch.empty_like(values)
+    if checked:
+        for t in (logp_smaller, logp_original, rewards, values):
+            assert t.shape == (n, b) and t.is_contiguous() and t.dtype == torch.float32 and t.is_cuda
+        assert bootstrap.shape == (b,) and bootstrap.is_contiguous() and bootstrap.dtype == torch.float32
+        assert discounts is None or (discounts.shape == (n, b) and discounts.is_contiguous())
+    vs, adv = (torch.empty_like(values), torch.empty_like(values)) if out is None else out
     _check(library().accerl_vtrace(logp_smaller.data_ptr(), logp_original.data_ptr(), rewards.data_ptr(),
                                    values.data_ptr(), bootstrap.data_ptr(),
                                    None if discounts is None else discounts.data_ptr(), n, b,
@@ -280,6 +284,10 @@ class Policy:
 
     def check(self):
         _check(library().accerl_policy_check(self._h))
+
+    def selftest_wait(self, poll_limit: int = 200, stream=0):
+        """accerl_policy_selftest_wait: makes a bounded device-side wait run out on purpose."""
+        _check(library().accerl_policy_selftest_wait(self._h, poll_limit, stream))
 
     def info(self, batch: int | None = None) -> dict:
         na, ws, nl = C.c_int32(), C.c_size_t(), C.c_int32()

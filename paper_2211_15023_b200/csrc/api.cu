@@ -386,7 +386,7 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         return ACCERL_ERR_INVALID_ARG;
     }
     if (flags & ~(uint32_t)(ACCERL_FLAG_KEEP_ACTIVATIONS | ACCERL_FLAG_FORCE_GENERIC | ACCERL_FLAG_TAP_FUSED |
-                            ACCERL_FLAG_VALUE_HEAD)) {
+                            ACCERL_FLAG_VALUE_HEAD | ACCERL_FLAG_TEST_NO_FASTDIV)) {
         set_error("create: unknown flag bits 0x%x", flags);
         return ACCERL_ERR_INVALID_ARG;
     }
@@ -872,6 +872,7 @@ accerl_status accerl_policy_info(const accerl_policy *p, int32_t batch, int32_t 
         s += line;
         ++launches;
     }
+    if (!p->plan_note.empty()) s += "note: " + p->plan_note + "\n";
     if (launches_per_act) *launches_per_act = launches;
     if (plan_buf && plan_buf_bytes) {
         size_t n = std::min(plan_buf_bytes - 1, s.size());

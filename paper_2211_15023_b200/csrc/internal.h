@@ -122,6 +122,7 @@ struct accerl_policy {
                                           // plan's sampler is a launch of its own and n_out != n_actions
     std::vector<accerl::LayerPlan> layers;
     std::vector<accerl::Step> steps;      // the launch sequence of one act call
+    std::string plan_note;                // why a faster plan was not taken (shown by accerl_policy_info)
     std::vector<accerl::TcStep> tc_steps;
     std::vector<accerl::PoolDualParams> pools;
     accerl::Conv1Params conv1 = {};       // used by a Step::CONV1_FRAMES launch

@@ -105,6 +105,7 @@ cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *
                                  cudaStream_t st);
 // exhaustive check of the three-step division against the IEEE divide for one output scale
 accerl_status verify_fastdiv(float s_out, float inv_s_out, bool relu, float y_max, bool *ok);
+accerl_status choose_fastdiv(float s_out, bool relu, float y_max, bool allow, float *inv_s_out, int *fast_div);
 bool fit_ingest_line(const int8_t *lut, uint32_t *mul, uint32_t *add);
 bool fit_ingest_float_line(const int8_t *lut, uint32_t mul, uint32_t add, uint32_t *a_bits, uint32_t *c1_bits);
 

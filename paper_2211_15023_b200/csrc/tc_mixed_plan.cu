@@ -731,19 +731,26 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                 kmax = std::max(kmax, d.s_in * d.s_w[c]);
                 bmax = std::max(bmax, fabsf(d.bias[c]));
             }
-            bool ok = false;
-            st = verify_fastdiv(g.s_out, g.inv_s_out, g.relu_out != 0, 2147483648.0f * kmax + bmax, &ok);
+            st = choose_fastdiv(g.s_out, g.relu_out != 0, 2147483648.0f * kmax + bmax,
+                                !(p->flags & ACCERL_FLAG_TEST_NO_FASTDIV), &g.inv_s_out, &g.fast_div);
             if (st != ACCERL_OK) return st;
-            g.fast_div = ok ? 1 : 0;
         }
         g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first) || hp_out) ? 1 : 0;
-        if (role[i] == TCPX && !g.fast_div) return bail();  // multi-pixel rows need the verified division
+        if (role[i] == TCPX && !g.fast_div) {  // multi-pixel rows need the verified division
+            p->plan_note = "tensor-core plan not used: the division-free requantiser could not be verified for the "
+                           "output scale of layer " + std::to_string(i);
+            return bail();
+        }
         if (hp_out) {
             g.hpool = 1;
             g.px_w = (L.out_w - 3) / 2 + 1;  // pooled width
         }
         if (role[i] == TCFIRST && hpool_first) {
-            if (!g.fast_div) return bail();
+            if (!g.fast_div) {
+                p->plan_note = "tensor-core plan not used: the division-free requantiser could not be verified for the "
+                               "output scale of layer " + std::to_string(i);
+                return bail();
+            }
             g.hpool = 1;
             g.px_per_row = 8;  // selects the multi-pixel kernel
             g.px_cols = d.out_c;

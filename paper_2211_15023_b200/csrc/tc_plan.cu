@@ -208,14 +208,14 @@ __global__ void verify_fastdiv_kernel(float s, float r, float y_max, unsigned lo
 accerl_status verify_fastdiv(float s_out, float inv_s_out, bool relu, float y_max, bool *ok)
 {
     struct Key {
-        float s, ymax;
+        float s, r, ymax;
         bool relu, ok;
     };
     static std::vector<Key> cache;
     static std::mutex mu;
     std::lock_guard<std::mutex> lock(mu);
     for (const Key &k : cache)
-        if (k.s == s_out && k.relu == relu && k.ymax >= y_max) {
+        if (k.s == s_out && k.r == inv_s_out && k.relu == relu && k.ymax >= y_max) {
             *ok = k.ok;
             return ACCERL_OK;
         }
@@ -235,7 +235,33 @@ accerl_status verify_fastdiv(float s_out, float inv_s_out, bool relu, float y_ma
         return ACCERL_ERR_CUDA;
     }
     *ok = host == 0;
-    cache.push_back(Key{s_out, y_max, relu, *ok});
+    cache.push_back(Key{s_out, inv_s_out, y_max, relu, *ok});
+    return ACCERL_OK;
+}
+
+// Reciprocal for the three-step division by s_out: fl(1 / s_out) or, where that one fails the
+// exhaustive comparison, one of its two neighbours (the correction step works with any reciprocal
+// that close; which rare operand patterns round wrongly differs between them).  *fast_div = 0 and
+// *inv_s_out = fl(1 / s_out) when none verifies or `allow` is false: the layer then runs the
+// epilogue with the exact fallback near ties, which assumes the correctly rounded reciprocal.
+accerl_status choose_fastdiv(float s_out, bool relu, float y_max, bool allow, float *inv_s_out, int *fast_div)
+{
+    volatile float inv = 1.0f / s_out;  // IEEE reciprocal, rounded once
+    const float r0 = inv;
+    *inv_s_out = r0;
+    *fast_div = 0;
+    if (!allow) return ACCERL_OK;
+    const float cand[3] = {r0, nextafterf(r0, 2.f * r0), nextafterf(r0, 0.f)};
+    for (float r : cand) {
+        bool ok = false;
+        accerl_status st = verify_fastdiv(s_out, r, relu, y_max, &ok);
+        if (st != ACCERL_OK) return st;
+        if (ok) {
+            *inv_s_out = r;
+            *fast_div = 1;
+            return ACCERL_OK;
+        }
+    }
     return ACCERL_OK;
 }
 
@@ -400,6 +426,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
             volatile float inv = 1.0f / L.s_out;  // IEEE reciprocal, rounded once
             g.inv_s_out = inv;
         }
+        const bool allow_fastdiv = !(p->flags & ACCERL_FLAG_TEST_NO_FASTDIV);
         if (!logits) {
             // largest |y| = |fma(acc, k, b)| the layer can produce: |acc| < 2^31
             float kmax = 0.f, bmax = 0.f;
@@ -407,11 +434,9 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 kmax = std::max(kmax, d.s_in * d.s_w[c]);
                 bmax = std::max(bmax, fabsf(d.bias[c]));
             }
-            bool ok = false;
-            accerl_status vs = verify_fastdiv(g.s_out, g.inv_s_out, g.relu_out != 0,
-                                              2147483648.0f * kmax + bmax, &ok);
+            accerl_status vs = choose_fastdiv(g.s_out, g.relu_out != 0, 2147483648.0f * kmax + bmax,
+                                              allow_fastdiv, &g.inv_s_out, &g.fast_div);
             if (vs != ACCERL_OK) return vs;
-            g.fast_div = ok ? 1 : 0;
         }
         g.split_cols = g.n_tile >= 128 ? 1 : 0;  // 128 / 256 columns: 32 / 64 per warpgroup
         g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;

@@ -57,26 +57,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 }
 
 // Bounded wait: gives up after kSpinPolls + kWaitLimitPolls polls or as soon as another role has
-// given up.  mbarrier.try_wait itself suspends the thread for a hardware-chosen interval, so the
-// first kSpinPolls polls follow each other directly: a hand-over between two roles then costs
-// the barrier's latency, not a sleep quantum (with 32..256 ns sleeps from the first miss on, every
-// hand-over of a pipeline lost up to half a microsecond).  Only a wait that lasts longer backs off
-// with pauses that double up to 256 ns, so that it does not take issue slots from working warps.
+// given up.  The pause between polls doubles up to 256 ns: a warp that waits for a whole tile must
+// not take issue slots from the working ones, one that waits briefly still wakes up quickly.
+// (mbarrier.try_wait itself suspends the thread for a hardware-chosen interval; polling it
+// kSpinPolls times before the first pause was measured with 0, 16, 128 and 2048 polls: no
+// difference on any layer, so the default is 0.)
 #ifndef ACCERL_SPIN_POLLS
-#define ACCERL_SPIN_POLLS 2048
+#define ACCERL_SPIN_POLLS 0
 #endif
 constexpr int kSpinPolls = ACCERL_SPIN_POLLS;
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          int *status, int code)
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                                  int *status, int code, int spin_polls, int sleep_polls)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    for (int i = 0; i < kSpinPolls; ++i) {
+    for (int i = 0; i < spin_polls; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63) == 63 && *abort_flag) return false;
     }
     unsigned ns = 32;
-    for (int i = 0; i < kWaitLimitPolls; ++i) {
+    for (int i = 0; i < sleep_polls; ++i) {
         __nanosleep(ns);
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
@@ -85,6 +85,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     atomicOr(status, code);
     return false;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          int *status, int code)
+{
+    return mbar_wait_limited(bar, parity, abort_flag, status, code, kSpinPolls, kWaitLimitPolls);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,

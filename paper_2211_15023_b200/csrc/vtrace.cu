@@ -28,18 +28,37 @@ vtrace_kernel(const float *__restrict__ logp_smaller, const float *__restrict__ 
     double v_next = (double)bootstrap[b];  // V(x_{t+1})
     double vs_next = v_next;               // v_{t+1}
     double carry = 0.0;                    // v_{t+1} - V(x_{t+1})
-    for (int t = n - 1; t >= 0; --t) {
-        const long long i = (long long)t * B + b;
-        const double ratio = exp((double)logp_original[i] - (double)logp_smaller[i]);
-        const double rho = fmin(ratio, (double)rho_hat), c = fmin(ratio, (double)c_hat);
-        const double g = discounts ? (double)discounts[i] : (double)gamma;
-        const double v = (double)values[i], r = (double)rewards[i];
-        const double delta = rho * (r + g * v_next - v);
-        carry = delta + g * c * carry;
-        if (adv) adv[i] = (float)(rho * (r + g * vs_next - v));
-        vs_next = v + carry;
-        vs[i] = (float)vs_next;
-        v_next = v;
+    // The recursion is sequential in t but its inputs are not: the loads of kChunk steps are issued
+    // together (a rollout is one thread, so nothing else hides the memory latency).
+    constexpr int kChunk = 8;
+    for (int t1 = n - 1; t1 >= 0; t1 -= kChunk) {
+        float lo[kChunk], ls[kChunk], rw[kChunk], vv[kChunk], dc[kChunk];
+#pragma unroll
+        for (int j = 0; j < kChunk; ++j) {
+            const int t = t1 - j;
+            const long long i = (long long)(t < 0 ? 0 : t) * B + b;
+            lo[j] = logp_original[i];
+            ls[j] = logp_smaller[i];
+            rw[j] = rewards[i];
+            vv[j] = values[i];
+            dc[j] = discounts ? discounts[i] : gamma;
+        }
+#pragma unroll
+        for (int j = 0; j < kChunk; ++j) {
+            const int t = t1 - j;
+            if (t < 0) break;
+            const long long i = (long long)t * B + b;
+            const double ratio = exp((double)lo[j] - (double)ls[j]);
+            const double rho = fmin(ratio, (double)rho_hat), c = fmin(ratio, (double)c_hat);
+            const double g = (double)dc[j];
+            const double v = (double)vv[j], r = (double)rw[j];
+            const double delta = rho * (r + g * v_next - v);
+            carry = delta + g * c * carry;
+            if (adv) adv[i] = (float)(rho * (r + g * vs_next - v));
+            vs_next = v + carry;
+            vs[i] = (float)vs_next;
+            v_next = v;
+        }
     }
 }
 
@@ -74,7 +93,7 @@ extern "C" accerl_status accerl_vtrace(const float *logp_smaller_dev, const floa
         set_error("vtrace: misaligned pointer (4 bytes needed)");
         return ACCERL_ERR_INVALID_ARG;
     }
-    const int threads = 128;
+    const int threads = batch >= 148 * 128 * 4 ? 128 : 32;  // few rollouts: spread them over the SMs
     vtrace_kernel<<<(unsigned)((batch + threads - 1) / threads), threads, 0, (cudaStream_t)cuda_stream>>>(
         logp_smaller_dev, logp_original_dev, rewards_dev, values_dev, bootstrap_dev, discounts_dev, n_steps,
         batch, gamma, rho_hat, c_hat, vs_dev, adv_dev);

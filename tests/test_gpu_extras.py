@@ -148,3 +148,26 @@ def test_mixing_of_two_policies(alpha):
         assert 0 < out["use_smaller"].sum() < b
     gs.close()
     go.close()
+
+
+def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_handle_usable():
+    """The give-up path of the bounded waits: a one-warp kernel waits, with a limit of a few hundred
+    polls, on a barrier nothing arrives at; the status word is set, check() reports TIMEOUT once,
+    and the next step runs and checks clean."""
+    import paper_2211_15023_b200 as P
+    name, b = "nature_cnn_b160", 16
+    pol = W.drawn_int8_policy(name)
+    g = P.Policy(pol, b)
+    obs, u = torch.from_numpy(W.observations(name, b)).cuda(), torch.from_numpy(W.uniforms(name, b)).cuda()
+    first = [t.clone() for t in g.act(obs, u)]
+    g.check()
+    g.selftest_wait(300)
+    with pytest.raises(P.AccerlError) as e:
+        g.check()
+    assert e.value.status == 6 and "0x80" in str(e.value)
+    g.check()  # the word was cleared
+    again = g.act(obs, u)
+    g.check()
+    for x, y in zip(first, again):
+        assert torch.equal(x, y)
+    g.close()
