@@ -137,6 +137,61 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
                                    int32_t device);
 
 /*
+ * One layer of an fp32 network, for accerl_policy_create_fp32: the fields of accerl_layer_desc
+ * without the quantisation results.  `w` is fp32 OIHW (FC: [out_c][in_c]), `bias` fp32 [out_c];
+ * both NULL for a max-pool.  All pointers are HOST pointers, copied during the call.
+ */
+typedef struct {
+    int32_t kind; /* accerl_layer_kind */
+    uint32_t flags;
+    int32_t in_c, in_h, in_w, out_c, kh, kw, stride, pad;
+    const float *w;
+    const float *bias;
+    int32_t skip_from; /* -1, or the earlier layer whose output is added into the accumulators */
+} accerl_layer_fp32;
+
+/*
+ * Post-training quantisation on the device, then accerl_policy_create (Section 2.2, paragraph
+ * "Parameter Quantization": the Compressor quantises the Learner's fp32 policy for the Actors;
+ * paragraph "Structured Pruning" for the optional pruning).  The scheme, each step on the GPU:
+ *   pruning (prune_2_4 != 0): of every four consecutive K positions, K = (kh, kw, c_in) with c_in
+ *       fastest, keep the two weights of largest magnitude (lower index wins a tie)
+ *   weights:     s_w[c] = max_k |w[c, k]| / 127 (1 for an all-zero channel);
+ *                q = clamp(rintf(w / s_w[c]), -127, 127)
+ *   input:       s_input = max |x| / 127 over the calibration batch (frames: x = u / 255)
+ *   activations: layer by layer, s_out = max |y| / 127 over the calibration batch, y the epilogue
+ *                float (after the residual add and the ReLU) computed from the already quantised
+ *                preceding layers; 1 if the maximum is 0; a max-pool passes its scale through;
+ *                the last layer has s_out = 1
+ *   residual:    skip_mul[c] = clamp(rintf(s_x / (s_in * s_w[c])), 0, 32767), s_x the scale of the
+ *                tensor that is added
+ * Every division is the IEEE fp32 one; maxima and integer sums do not depend on evaluation order,
+ * so the result is the same bits on every run.
+ *   calib_obs_host  host, calib_rows observations in the layout `act` takes (uint8 [rows, C, H, W]
+ *                   or fp32 [rows, D])
+ *   the other arguments are those of accerl_policy_create; ACCERL_FLAG_VALUE_HEAD as there
+ * Create-time work with plain kernels (tens of milliseconds for a thousand frames); transient
+ * device memory: the calibration batch's int8 activations plus one int32 tensor of the largest
+ * layer output.  Errors: INVALID_ARG, UNSUPPORTED, OOM, CUDA; *out is NULL then.
+ */
+accerl_status accerl_policy_create_fp32(accerl_policy **out, int32_t in_kind, const int32_t in_shape[3],
+                                        const accerl_layer_fp32 *layers, int32_t n_layers,
+                                        const void *calib_obs_host, int32_t calib_rows,
+                                        int32_t prune_2_4, int32_t max_batch, uint32_t flags,
+                                        int32_t device);
+
+/*
+ * Read back what accerl_policy_create_fp32 computed for one layer (for storing the quantised
+ * policy, or for checking it): int8 weights in OIHW order, per-channel weight scales, residual
+ * multipliers, and the layer's input / output activation scales.  Any output pointer may be NULL;
+ * w_bytes is the size of w_host.  A max-pool has no weights (nothing is written for it).
+ * Errors: INVALID_ARG (also for a handle not built by accerl_policy_create_fp32).
+ */
+accerl_status accerl_policy_export(const accerl_policy *p, int32_t layer, int8_t *w_host,
+                                   size_t w_bytes, float *s_w_host, int32_t *skip_mul_host,
+                                   float *s_in_out, float *s_out_out);
+
+/*
  * One Actor step for a batch of states (Introduction, Fig. 1 "Agent"; Section 2.3, Eq. V-trace
  * for the behaviour log-probability): quantise the observations, run every layer, sample.
  *   obs_dev       device, uint8 [batch, C, H, W] or fp32 [batch, D]; 16-byte aligned; read only

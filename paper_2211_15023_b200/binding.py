@@ -36,6 +36,14 @@ class LayerDesc(C.Structure):
                 ("skip_from", C.c_int32), ("skip_mul", C.c_void_p)]
 
 
+class LayerFp32(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("flags", C.c_uint32),
+                ("in_c", C.c_int32), ("in_h", C.c_int32), ("in_w", C.c_int32),
+                ("out_c", C.c_int32), ("kh", C.c_int32), ("kw", C.c_int32),
+                ("stride", C.c_int32), ("pad", C.c_int32),
+                ("w", C.c_void_p), ("bias", C.c_void_p), ("skip_from", C.c_int32)]
+
+
 def library_path() -> str:
     return os.path.join(_HERE, "libaccerl.so")
 
@@ -66,6 +74,11 @@ def library() -> C.CDLL:
         lib.accerl_vtrace.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, f32, vp, vp, vp]
         for f in ("accerl_policy_act_ex", "accerl_policy_kl", "accerl_policy_act_mixed", "accerl_vtrace"):
             getattr(lib, f).restype = C.c_int
+        lib.accerl_policy_create_fp32.argtypes = [C.POINTER(vp), i32, C.POINTER(i32), C.POINTER(LayerFp32), i32, vp,
+                                                  i32, i32, i32, C.c_uint32, i32]
+        lib.accerl_policy_create_fp32.restype = C.c_int
+        lib.accerl_policy_export.argtypes = [vp, i32, vp, C.c_size_t, vp, vp, C.POINTER(f32), C.POINTER(f32)]
+        lib.accerl_policy_export.restype = C.c_int
         lib.accerl_policy_selftest_wait.argtypes = [vp, i32, vp]
         lib.accerl_policy_selftest_wait.restype = C.c_int
         lib.accerl_tc_probe_i8.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32, C.POINTER(f32), C.POINTER(f32)]
@@ -167,6 +180,57 @@ class Policy:
     relu_in, relu_out, logits, skip_from, s_in, s_out and numpy arrays w (int8 OIHW), s_w, bias,
     skip_mul (or None).
     """
+
+    @classmethod
+    def from_fp32(cls, in_kind: str, in_shape, layers, params, calib_obs, max_batch: int,
+                  prune24: bool = False, flags: int = 0, device: int = 0) -> "Policy":
+        """accerl_policy_create_fp32: quantise and calibrate on the device.  ``layers`` are
+        architecture dicts, ``params`` the matching fp32 {w, bias} (None for max-pool)."""
+        lib = library()
+        self = cls.__new__(cls)
+        self._h = C.c_void_p()
+        n = len(layers)
+        descs = (LayerFp32 * n)()
+        keep = []
+        for i, (l, pr) in enumerate(zip(layers, params)):
+            d = descs[i]
+            d.kind = _KINDS[l["kind"]]
+            d.flags = (RELU_IN if l["relu_in"] else 0) | (RELU_OUT if l["relu_out"] else 0) | \
+                (LOGITS if l["logits"] else 0)
+            for k in ("in_c", "in_h", "in_w", "out_c", "kh", "kw", "stride", "pad", "skip_from"):
+                setattr(d, k, int(l[k]))
+            if pr is not None:
+                w, b = np.ascontiguousarray(pr["w"], np.float32), np.ascontiguousarray(pr["bias"], np.float32)
+                keep += [w, b]
+                d.w, d.bias = w.ctypes.data, b.ctypes.data
+        shape = (C.c_int32 * 3)(*[int(v) for v in in_shape])
+        calib = np.ascontiguousarray(calib_obs, np.uint8 if in_kind == "u8" else np.float32)
+        self.layers = [dict(l) for l in layers]
+        self.in_kind, self.in_shape = in_kind, tuple(int(v) for v in in_shape)
+        self.max_batch, self.device = int(max_batch), int(device)
+        self.value_head = bool(layers[-1].get("value"))
+        if self.value_head:
+            flags = int(flags) | FLAG_VALUE_HEAD
+        _check(lib.accerl_policy_create_fp32(C.byref(self._h), 0 if in_kind == "u8" else 1, shape, descs, n,
+                                             calib.ctypes.data, int(calib.shape[0]), int(bool(prune24)),
+                                             self.max_batch, int(flags), self.device))
+        self.n_actions = int(layers[-1]["out_c"]) - (1 if self.value_head else 0)
+        return self
+
+    def export(self, layer: int) -> dict:
+        """accerl_policy_export: the quantised parameters of one layer of a from_fp32 policy."""
+        l = self.layers[layer]
+        s_in, s_out = C.c_float(), C.c_float()
+        if l["kind"] == "maxpool":
+            _check(library().accerl_policy_export(self._h, layer, None, 0, None, None, C.byref(s_in), C.byref(s_out)))
+            return dict(w=None, s_w=None, skip_mul=None, s_in=np.float32(s_in.value), s_out=np.float32(s_out.value))
+        w = np.empty((l["out_c"], l["in_c"], l["kh"], l["kw"]), np.int8)
+        s_w = np.empty(l["out_c"], np.float32)
+        sm = np.empty(l["out_c"], np.int32) if l["skip_from"] >= 0 else None
+        _check(library().accerl_policy_export(self._h, layer, w.ctypes.data, w.nbytes, s_w.ctypes.data,
+                                              None if sm is None else sm.ctypes.data, C.byref(s_in),
+                                              C.byref(s_out)))
+        return dict(w=w, s_w=s_w, skip_mul=sm, s_in=np.float32(s_in.value), s_out=np.float32(s_out.value))
 
     def __init__(self, policy: dict, max_batch: int, flags: int = 0, device: int = 0):
         lib = library()

@@ -151,6 +151,14 @@ struct accerl_policy {
     void *st_obs = nullptr;
     float *st_u = nullptr, *st_logits = nullptr, *st_logp = nullptr;
     int32_t *st_actions = nullptr;
+    // the quantised parameters accerl_policy_create_fp32 computed (empty for other handles)
+    struct PtqLayer {
+        std::vector<int8_t> w;
+        std::vector<float> s_w;
+        std::vector<int32_t> skip_mul;
+        float s_in = 1.f, s_out = 1.f;
+    };
+    std::vector<PtqLayer> ptq;
     // outputs of this policy inside accerl_policy_act_mixed (allocated on its first call)
     float *mix_logits = nullptr, *mix_logp = nullptr, *mix_value = nullptr, *mix_entropy = nullptr;
     int32_t *mix_actions = nullptr;

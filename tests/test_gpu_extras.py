@@ -171,3 +171,36 @@ def test_a_wait_that_runs_out_reports_timeout_and_leaves_the_handle_usable():
     for x, y in zip(first, again):
         assert torch.equal(x, y)
     g.close()
+
+
+@pytest.mark.parametrize("name,rows", [("cartpole_mlp", 256), ("lunarlander_mlp", 300), ("nature_cnn_b160", 48),
+                                       ("student_cnn_b8192", 40), ("impala_resnet_b16384", 12)])
+def test_quantisation_and_calibration_on_the_device(name, rows):
+    """accerl_policy_create_fp32 against the oracle's quantiser and calibrator: int8 weights (2:4
+    pruned for the residual network), weight scales, every activation scale and the residual
+    multipliers must be the same bits, and the policy built from them must act like the oracle's."""
+    import paper_2211_15023_b200 as P
+    c = W.config(name)
+    params = W.fp32_parameters(name)
+    calib = W.calibration_batch(name, rows)
+    want = oracle.calibrate(c["in_kind"], c["in_shape"], c["layers"], params, calib, c["prune24"])
+    b = 19
+    g = P.Policy.from_fp32(c["in_kind"], c["in_shape"], c["layers"], params, calib, b, prune24=c["prune24"])
+    for i, l in enumerate(want["layers"]):
+        got = g.export(i)
+        assert got["s_in"] == np.float32(l["s_in"]) and got["s_out"] == np.float32(l["s_out"]), (i, got["s_in"], l["s_in"], got["s_out"], l["s_out"])
+        if l["kind"] == "maxpool":
+            continue
+        assert np.array_equal(got["w"], l["w"]), "layer %d: int8 weights differ" % i
+        assert np.array_equal(got["s_w"], l["s_w"]), "layer %d: weight scales differ" % i
+        if l["skip_from"] >= 0:
+            assert np.array_equal(got["skip_mul"], l["skip_mul"]), "layer %d: residual multipliers differ" % i
+        if c["prune24"]:
+            k = got["w"].transpose(0, 2, 3, 1).reshape(got["w"].shape[0], -1, 4)
+            assert ((k != 0).sum(-1) <= 2).all()
+    obs, u = W.observations(name, b), W.uniforms(name, b)
+    ref = oracle.forward(want, obs, u, keep=False)
+    out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+    g.check()
+    compare(ref, *out)
+    g.close()
