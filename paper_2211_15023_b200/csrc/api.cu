@@ -310,6 +310,11 @@ static accerl_status run_steps(accerl_policy *p, const void *obs_dev, const floa
             }
             ACCERL_CUDA_TRY(conv1_launch(p->conv1_map_b, p->conv1, B, (const uint8_t *)obs_dev, p->sm_count, st));
             break;
+        case Step::CONV_ROWS: {
+            const ConvRowsStep &cs = p->conv_rows[s.tc];
+            ACCERL_CUDA_TRY(conv_rows_launch(cs.map_a, cs.map_b, cs.prm, B, p->sm_count, st));
+            break;
+        }
         case Step::INGEST_NHWC4:
             ACCERL_CUDA_TRY(launch_ingest_u8_nhwc4((const uint8_t *)obs_dev, p->lut,
                                                    p->bufs[p->layers[0].in_buf].ptr, B, p->in_h,

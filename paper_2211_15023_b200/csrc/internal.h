@@ -9,6 +9,7 @@
 #include <vector>
 
 #include "accerl.h"
+#include "tc_conv.h"
 #include "tc_conv1.h"
 #include "tc_gemm.h"
 
@@ -52,9 +53,9 @@ struct LayerPlan {
 // ("ingest", "layer 3", "layers 3-4", "sample", joined by '+').
 struct Step {
     enum Kind { INGEST, CONV_GENERIC, FC_GENERIC, POOL_GENERIC, SAMPLE, INGEST_S2D, TC_GEMM, MLP_FUSED,
-                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4, FC_SAMPLE, CONV1_FRAMES } kind;
+                INGEST_NHWC4, POOL_DUAL, INGEST_PAD4, FC_SAMPLE, CONV1_FRAMES, CONV_ROWS } kind;
     int layer = -1;
-    int tc = -1;  // index into accerl_policy::tc_steps (TC_GEMM) or ::pools (POOL_DUAL)
+    int tc = -1;  // index into accerl_policy::tc_steps (TC_GEMM), ::pools (POOL_DUAL) or ::conv_rows (CONV_ROWS)
     std::string kernel, covers;
 };
 
@@ -65,6 +66,13 @@ struct TcStep {
     alignas(64) unsigned char map_b[128];
     TcGemmParams prm;
     bool resident_b = false;
+};
+
+// One launch of the strided-conv kernel (tc_conv.cu)
+struct ConvRowsStep {
+    alignas(64) unsigned char map_a[128];
+    alignas(64) unsigned char map_b[128];
+    ConvRowsParams prm;
 };
 
 struct MlpFusedParams;  // mlp_fused.cu
@@ -125,6 +133,7 @@ struct accerl_policy {
     std::string plan_note;                // why a faster plan was not taken (shown by accerl_policy_info)
     std::vector<accerl::TcStep> tc_steps;
     std::vector<accerl::PoolDualParams> pools;
+    std::vector<accerl::ConvRowsStep> conv_rows;
     accerl::Conv1Params conv1 = {};       // used by a Step::CONV1_FRAMES launch
     alignas(64) unsigned char conv1_map_b[128] = {};
     int8_t *in_pad4 = nullptr;            // frames as [n][H+2][PW][4] with the image at (1, 4)

@@ -531,6 +531,53 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 continue;
             }
         }
+        // Other strided convs on small grids with 48 or 64 output channels: the kernel with tiles of
+        // whole grid rows (tc_conv.cu); the un-fused tap plan keeps the general kernel as cross-check.
+        // (Measured at batch 8192: 64 channels 42.0 -> 39.9 and 37.9 -> 35.8 us for the second and
+        // third layer; with 32 channels the general kernel is the faster one, 27.6 against 29.7 us.)
+        if (d.kind == ACCERL_CONV2D && i > 0 && g.shifted && ts.resident_b && g.fast_div && !unfuse_for_taps(p) &&
+            n_total > 32 && n_total <= 64) {
+            ConvRowsStep cs;
+            if (conv_rows_plan(g.rows_per_image / g.grid_w, g.grid_w, g.chunk_bytes, d.kh / d.stride, n_total,
+                               p->max_batch, &cs.prm)) {
+                ConvRowsParams &c2 = cs.prm;
+                c2.out = g.out;
+                c2.out_h = g.out_h;
+                c2.out_w = g.out_w;
+                c2.out_s2d_log2 = g.out_s2d_log2;
+                c2.out_rows_per_image = g.out_rows_per_image;
+                c2.out_grid_w = g.out_grid_w;
+                c2.out_pitch = g.out_pitch;
+                c2.n_total = n_total;
+                c2.s_out = g.s_out;
+                c2.inv_s_out = g.inv_s_out;
+                c2.relu = g.relu_out;
+                c2.status = p->status_word;
+                for (int c = 0; c < d.out_c; ++c) {
+                    volatile float k = d.s_in * d.s_w[c];  // one fp32 rounding, never contracted
+                    c2.ks[c] = k;
+                    c2.bs[c] = d.bias[c];
+                }
+                void *w2_dev = nullptr;
+                accerl_status st2 = upload_bytes(p, packed.data(), packed.size(), &w2_dev);
+                if (st2 != ACCERL_OK) return st2;
+                st2 = tc_make_map(cs.map_a, p->bufs[L.in_buf].ptr, (long long)p->max_batch * rows_in_per_image,
+                                  row_bytes, row_bytes, c2.box_rows, row_bytes);
+                if (st2 != ACCERL_OK) return st2;
+                st2 = tc_make_map(cs.map_b, w2_dev, (long long)g.n_chunks * n_total, row_bytes, row_bytes, n_total,
+                                  row_bytes);
+                if (st2 != ACCERL_OK) return st2;
+                p->conv_rows.push_back(cs);
+                Step s;
+                s.kind = Step::CONV_ROWS;
+                s.layer = i;
+                s.tc = (int)p->conv_rows.size() - 1;
+                s.kernel = "conv_rows_kernel[3-step divide verified]";
+                s.covers = "layer " + std::to_string(i);
+                steps.push_back(s);
+                continue;
+            }
+        }
         if (!g.fuse_ingest && !tc_choose_pipeline(g, ts.resident_b)) {
             ts.resident_b = false;
             g.shifted = 0;
@@ -539,6 +586,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 p->tensor_s2d.assign(n_layers + 1, 1);
                 p->tap_missing.assign(n_layers + 1, 0);
                 p->tc_steps.clear();
+                p->conv_rows.clear();
                 return ACCERL_OK;
             }
         }
