@@ -340,6 +340,38 @@ def test_first_conv_kernel_other_frames_and_input_tables(hw, c1, peak):
         g.close()
 
 
+@pytest.mark.parametrize("hw,c2,c3", [((68, 100), 64, 48), ((52, 84), 64, 48), ((100, 52), 64, 64)],
+                         ids=["68x100_64_48", "52x84_64_48", "100x52_64_64"])
+def test_strided_conv_kernel_other_grids_and_widths(hw, c2, c3):
+    """The strided-conv kernel with tiles of whole grid rows on grids other than the Atari network's
+    (widths that leave idle rows in a tile, 48 and 64 output channels, 128- and 64-byte rows, 2 x 2
+    and 3 x 3 taps), small and ragged batches, with and without taps, against the un-fused plan's
+    general kernel and the oracle."""
+    import paper_2211_15023_b200 as P
+    H, Wd = hw
+    rng = np.random.default_rng(H * 7 + Wd + c2)
+    h1, w1 = (H - 8) // 4 + 1, (Wd - 8) // 4 + 1
+    h2, w2 = (h1 - 4) // 2 + 1, (w1 - 4) // 2 + 1
+    h3, w3 = h2 - 2, w2 - 2
+    layers = [W._conv(4, H, Wd, 32, 8, 4, 0), W._conv(32, h1, w1, c2, 4, 2, 0), W._conv(c2, h2, w2, c3, 3, 1, 0),
+              W._fc(c3 * h3 * w3, 64), W._fc(64, 5, relu_out=False, logits=True)]
+    params = W.parameters_for(layers, 13)
+    calib = rng.integers(0, 256, (16, 4, H, Wd), dtype=np.uint8)
+    pol = oracle.calibrate("u8", (4, H, Wd), layers, params, calib)
+    for b in (1, 29):
+        obs = rng.integers(0, 256, (b, 4, H, Wd), dtype=np.uint8)
+        u = rng.random(b, dtype=np.float32)
+        ref = oracle.forward(pol, obs, u)
+        for flags in (0, 5, 1):
+            g = P.Policy(pol, b, flags=flags)
+            plan = g.info()["plan"]
+            assert (plan.count("conv_rows_kernel") == 2) == (flags != 1), plan
+            out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+            g.check()
+            compare(ref, *out, taps=g.read_activation if flags else None)
+            g.close()
+
+
 def test_exact_ties_on_the_tensor_core_path():
     """Power-of-two scales make many epilogue quotients land exactly on k + 0.5: the requantiser
     must round them to even exactly as the IEEE divide + rintf of the definition does."""
