@@ -9,8 +9,10 @@
 //   (row, X) of every tile, its output address costs two multiplies per tile;
 // - a pipeline step is T tiles whose operand block (the T * S grid rows and the t - 1 rows the taps
 //   reach into) arrives by a few TMA boxes issued by one warp; kStages2 blocks are in flight;
-// - two warps issue the MMAs (descriptors computed in registers), sixteen warps drain
-//   accumulators; scales and biases are kernel parameters read from the constant bank, because
+// - four warps issue the MMAs, tiles in turn (descriptors computed in registers; one warp that
+//   shares its scheduler with five others issues an instruction every six to eight cycles, and a
+//   tile takes some two hundred: measured 49 / 41 / 36 us for the layer with one / two / four
+//   issuing warps), sixteen warps drain accumulators; scales and biases are kernel parameters read from the constant bank, because
 //   shared-memory loads of the epilogue queue behind the operand reads of the MMAs.
 //
 // Every wait is bounded; a wait that gives up sets the status word and all roles leave.
@@ -27,9 +29,9 @@ namespace accerl {
 
 namespace {
 
-constexpr int kMmaWarps2 = 2;
-constexpr int kEpiWarps2 = 16;
-constexpr int kWarps2 = 4 + kEpiWarps2;  // warps 0, 1 issue, warp 2 loads, warp 3 idles
+constexpr int kMmaWarps2 = 4;            // warps 0..3 issue MMAs, the CTA's tiles in turn
+constexpr int kEpiWarps2 = 16;           // warps 4..19 drain accumulators
+constexpr int kWarps2 = 4 + kEpiWarps2 + 1;  // the last warp issues the TMA loads
 constexpr int kThreads2 = 32 * kWarps2;
 constexpr int kStages2 = 3;
 constexpr int kMaxSlots2 = 16;
@@ -120,9 +122,10 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t st_lo = ((smem_u32(stages) + (uint32_t)(s * stage_bytes)) >> 4) | lo_flags;
-            for (int i = warp; i < T && ok; i += kMmaWarps2) {
+            for (int i = 0; i < T && ok; ++i) {
                 if (step * T + i >= p.total_tiles) break;
                 const int seq = k * T + i, slot = seq % kAccSlots;  // the CTA's tiles in order
+                if (seq % kMmaWarps2 != warp) continue;
                 ok = mbar_wait(acc_empty0 + 8 * slot, (uint32_t)(((seq / kAccSlots) & 1) ^ 1), abort_flag, p.status, 4);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -148,7 +151,7 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             if (ok && elect_one()) mma_commit(empty0 + 8 * s);  // the block is free when these MMAs retire
             __syncwarp();
         }
-    } else if (warp == 2) {
+    } else if (warp == kWarps2 - 1) {
         // ------------------------------------------------------------------ TMA producer
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the activations are the previous launch's output
         bool ok = true;
@@ -167,7 +170,7 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
             __syncwarp();
         }
-    } else if (warp >= 4) {
+    } else {
         // ------------------------------------------------------------------ epilogue
         const int ew = warp - 4, wg = ew >> 2, q = warp & 3;
         constexpr int kGroups = kEpiWarps2 / 4;

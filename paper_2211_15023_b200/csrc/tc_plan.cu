@@ -533,8 +533,8 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         }
         // Other strided convs on small grids with 48 or 64 output channels: the kernel with tiles of
         // whole grid rows (tc_conv.cu); the un-fused tap plan keeps the general kernel as cross-check.
-        // (Measured at batch 8192: 64 channels 42.0 -> 39.9 and 37.9 -> 35.8 us for the second and
-        // third layer; with 32 channels the general kernel is the faster one, 27.6 against 29.7 us.)
+        // (Measured at batch 8192: 64 channels 42.0 -> 36.5 and 37.9 -> 35.8 us for the second and
+        // third layer; with 32 channels the general kernel is as fast or faster, 26.6 against 28.7 us.)
         if (d.kind == ACCERL_CONV2D && i > 0 && g.shifted && ts.resident_b && g.fast_div && !unfuse_for_taps(p) &&
             n_total > 32 && n_total <= 64) {
             ConvRowsStep cs;
