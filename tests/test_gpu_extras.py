@@ -204,3 +204,20 @@ def test_quantisation_and_calibration_on_the_device(name, rows):
     g.check()
     compare(ref, *out)
     g.close()
+
+
+def test_tensor_pipe_probe_reports_plausible_costs_and_rejects_bad_arguments():
+    """accerl_tc_probe_i8: an N = 256 MMA is bound by its multiply-accumulates (8192 per cycle and
+    SM: 128 cycles), a narrow one by reading its operands from shared memory (about 40 cycles);
+    layout and row shift of the operands must not matter; bad arguments are refused on the host."""
+    import paper_2211_15023_b200 as P
+    wide = P.tc_probe_i8(256, 2, 2048, 148)
+    assert 120 <= wide["cycles_per_mma"] <= 140 and wide["tops"] > 3000, wide
+    narrow = P.tc_probe_i8(32, 1, 2048, 148)
+    assert 35 <= narrow["cycles_per_mma"] <= 50, narrow
+    shifted = P.tc_probe_i8(32, 1, 2048, 8, 64, 21, 8)
+    assert abs(shifted["cycles_per_mma"] - narrow["cycles_per_mma"]) < 3, (shifted, narrow)
+    for bad in ((24, 1, 2048, 1), (256, 4, 2048, 1), (32, 1, 2050, 1), (32, 5, 2048, 1), (32, 1, 2048, 1, 48)):
+        with pytest.raises(P.AccerlError) as e:
+            P.tc_probe_i8(*bad)
+        assert e.value.status == 1
