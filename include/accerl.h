@@ -349,8 +349,10 @@ accerl_status accerl_policy_act_noalloc(accerl_policy *p, const void *obs_dev,
  * environments on the CPU, Section 2.1): copies obs and uniforms to device staging buffers owned
  * by the handle, runs accerl_policy_act, copies the three results back and waits for them.
  * All five pointers are host pointers (pinned memory makes the copies asynchronous and faster;
- * pageable memory works).  The staging buffers are allocated on the first call.  Blocks until
- * the results are in the host buffers.
+ * pageable memory works).  The staging buffers are allocated on the first call.  Batches of 4096
+ * states and more go in eight chunks whose host->device copies run on a stream of the handle's own
+ * while the previous chunk computes on `cuda_stream`; the results are those of one call on the
+ * whole batch.  Blocks until the results are in the host buffers.
  */
 accerl_status accerl_policy_act_host(accerl_policy *p, const void *obs_host,
                                      const float *uniforms_host, int32_t batch,

@@ -364,6 +364,8 @@ void accerl_policy_destroy(accerl_policy *p)
     cudaDeviceSynchronize();
     for (void *d : p->owned) cudaFree(d);
     for (cudaEvent_t ev : p->events) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : p->copy_events) cudaEventDestroy(ev);
+    if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
     delete p;
 }
 
@@ -744,15 +746,59 @@ accerl_status accerl_policy_act_host(accerl_policy *p, const void *obs_host,
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const size_t B = (size_t)batch;
-    ACCERL_CUDA_TRY(cudaMemcpyAsync(p->st_obs, obs_host, obs_per_state * B, cudaMemcpyHostToDevice, st));
-    ACCERL_CUDA_TRY(cudaMemcpyAsync(p->st_u, uniforms_host, 4 * B, cudaMemcpyHostToDevice, st));
-    accerl_status s = accerl_policy_act(p, p->st_obs, p->st_u, batch, p->st_logits, p->st_actions,
-                                        p->st_logp, cuda_stream);
-    if (s != ACCERL_OK) return s;
-    ACCERL_CUDA_TRY(cudaMemcpyAsync(logits_host, p->st_logits, 4 * B * p->n_actions,
-                                    cudaMemcpyDeviceToHost, st));
-    ACCERL_CUDA_TRY(cudaMemcpyAsync(actions_host, p->st_actions, 4 * B, cudaMemcpyDeviceToHost, st));
-    ACCERL_CUDA_TRY(cudaMemcpyAsync(logp_host, p->st_logp, 4 * B, cudaMemcpyDeviceToHost, st));
+    // Large batches go in chunks: the host->device copy of chunk i + 1 runs on a stream of its own
+    // while chunk i computes (the copy is PCIe-bound and by far the longer part; the chunks only
+    // hide the compute and the copies back behind it).  States are independent, so the results are
+    // those of one call on the whole batch.
+    const int n_chunks = batch >= 4096 ? 8 : 1;
+    if (n_chunks > 1 && !p->copy_stream) {
+        ACCERL_CUDA_TRY(cudaStreamCreateWithFlags(&p->copy_stream, cudaStreamNonBlocking));
+        for (int i = 0; i < 9; ++i) {
+            cudaEvent_t ev;
+            ACCERL_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+            p->copy_events.push_back(ev);
+        }
+    }
+    if (n_chunks == 1) {
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(p->st_obs, obs_host, obs_per_state * B, cudaMemcpyHostToDevice, st));
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(p->st_u, uniforms_host, 4 * B, cudaMemcpyHostToDevice, st));
+        accerl_status s = accerl_policy_act(p, p->st_obs, p->st_u, batch, p->st_logits, p->st_actions,
+                                            p->st_logp, cuda_stream);
+        if (s != ACCERL_OK) return s;
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(logits_host, p->st_logits, 4 * B * p->n_actions,
+                                        cudaMemcpyDeviceToHost, st));
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(actions_host, p->st_actions, 4 * B, cudaMemcpyDeviceToHost, st));
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(logp_host, p->st_logp, 4 * B, cudaMemcpyDeviceToHost, st));
+        ACCERL_CUDA_TRY(cudaStreamSynchronize(st));
+        return ACCERL_OK;
+    }
+    // the staging buffers may still be read by earlier work of the caller's stream
+    ACCERL_CUDA_TRY(cudaEventRecord(p->copy_events[8], st));
+    ACCERL_CUDA_TRY(cudaStreamWaitEvent(p->copy_stream, p->copy_events[8], 0));
+    const size_t per = ((B + n_chunks - 1) / n_chunks + 15) & ~(size_t)15;  // keeps every chunk 16-byte aligned
+    const size_t A = (size_t)p->n_actions;
+    int used = 0;
+    for (size_t b0 = 0; b0 < B; b0 += per, ++used) {
+        const size_t nb = std::min(per, B - b0);
+        ACCERL_CUDA_TRY(cudaMemcpyAsync((char *)p->st_obs + b0 * obs_per_state, (const char *)obs_host + b0 * obs_per_state,
+                                        obs_per_state * nb, cudaMemcpyHostToDevice, p->copy_stream));
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(p->st_u + b0, uniforms_host + b0, 4 * nb, cudaMemcpyHostToDevice, p->copy_stream));
+        ACCERL_CUDA_TRY(cudaEventRecord(p->copy_events[used], p->copy_stream));
+    }
+    used = 0;
+    for (size_t b0 = 0; b0 < B; b0 += per, ++used) {
+        const size_t nb = std::min(per, B - b0);
+        ACCERL_CUDA_TRY(cudaStreamWaitEvent(st, p->copy_events[used], 0));
+        accerl_status s = accerl_policy_act(p, (const char *)p->st_obs + b0 * obs_per_state, p->st_u + b0, (int32_t)nb,
+                                            p->st_logits + b0 * A, p->st_actions + b0, p->st_logp + b0, cuda_stream);
+        if (s != ACCERL_OK) {
+            cudaStreamSynchronize(p->copy_stream);
+            return s;
+        }
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(logits_host + b0 * A, p->st_logits + b0 * A, 4 * nb * A, cudaMemcpyDeviceToHost, st));
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(actions_host + b0, p->st_actions + b0, 4 * nb, cudaMemcpyDeviceToHost, st));
+        ACCERL_CUDA_TRY(cudaMemcpyAsync(logp_host + b0, p->st_logp + b0, 4 * nb, cudaMemcpyDeviceToHost, st));
+    }
     ACCERL_CUDA_TRY(cudaStreamSynchronize(st));
     return ACCERL_OK;
 }

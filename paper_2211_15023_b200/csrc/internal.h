@@ -160,6 +160,8 @@ struct accerl_policy {
     void *st_obs = nullptr;
     float *st_u = nullptr, *st_logits = nullptr, *st_logp = nullptr;
     int32_t *st_actions = nullptr;
+    cudaStream_t copy_stream = nullptr;   // host->device copies of chunked accerl_policy_act_host calls
+    std::vector<cudaEvent_t> copy_events; // one per chunk, and one for the caller's stream
     // the quantised parameters accerl_policy_create_fp32 computed (empty for other handles)
     struct PtqLayer {
         std::vector<int8_t> w;

@@ -125,6 +125,27 @@ def test_act_host_matches_device_call():
     g.close()
 
 
+def test_act_host_in_chunks_matches_device_call():
+    """From 4096 states on the host-buffer call goes in eight chunks with the copies overlapped; a
+    batch that does not divide evenly (4099 on the MLP, whose fp32 rows keep every chunk aligned)
+    and two calls in a row must give what one device call gives."""
+    import paper_2211_15023_b200 as P
+    name, b = "lunarlander_mlp", 4099
+    pol = calibrated(name)
+    g = P.Policy(pol, b)
+    for call in range(2):
+        obs, u = W.observations(name, b, seed=call), W.uniforms(name, b, seed=10 + call)
+        dev = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        host = (torch.empty((b, 4), dtype=torch.float32).pin_memory(),
+                torch.empty(b, dtype=torch.int32).pin_memory(),
+                torch.empty(b, dtype=torch.float32).pin_memory())
+        g.act_host(torch.from_numpy(obs).pin_memory(), torch.from_numpy(u).pin_memory(), host)
+        for x, y in zip(dev, host):
+            assert np.array_equal(x, y.numpy())
+    g.check()
+    g.close()
+
+
 def test_saturating_inputs_and_extreme_uniforms():
     import paper_2211_15023_b200 as P
     name = "lunarlander_mlp"
