@@ -46,7 +46,10 @@ struct __align__(8) Bars2 {
 
 }  // namespace
 
-template <int NCOLS>
+// TAPS_T / RB_T: taps per side and bytes of an operand row as compile-time constants (0 = taken from
+// the parameters); with them the issue loop of a tile is straight-line code, and the issuing warps'
+// instruction count is what bounds how fast tiles start.
+template <int NCOLS, int TAPS_T, int RB_T>
 __global__ void __launch_bounds__(kThreads2, 1)
 conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ ConvRowsParams p)
@@ -57,7 +60,7 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int kSlotCols = NCOLS <= 32 ? 32 : 64;     // tensor-memory columns of one accumulator
     constexpr int kAccSlots = 512 / kSlotCols;
-    const int RB = p.row_bytes, taps = p.taps, n_taps = taps * taps;
+    const int RB = RB_T ? RB_T : p.row_bytes, taps = TAPS_T ? TAPS_T : p.taps, n_taps = taps * taps;
     const int b_bytes = n_taps * NCOLS * RB;
     uint8_t *b_tiles = smem;
     uint8_t *stages = smem + ((b_bytes + 1023) & ~1023);
@@ -132,16 +135,29 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (elect_one()) {
                     const uint32_t d = tmem_base + (uint32_t)(slot * kSlotCols);
                     const uint32_t a_tile = st_lo + (uint32_t)(i * S * Ws) * row16;
-                    uint32_t b_j = b_lo, first = 0;
-                    for (int ty = 0; ty < taps; ++ty) {
-                        uint32_t a_j = a_tile + (uint32_t)(ty * Ws) * row16;
-                        for (int tx = 0; tx < taps; ++tx) {
-                            for (uint32_t ks = 0; ks < ksteps; ++ks) {
-                                mma_i8(d, desc_hi | (a_j + 2 * ks), desc_hi | (b_j + 2 * ks), idesc, first);
-                                first = 1;
+                    if constexpr (TAPS_T != 0 && RB_T != 0) {
+                        const uint32_t a_row = (uint32_t)Ws * row16;
+#pragma unroll
+                        for (int ty = 0; ty < TAPS_T; ++ty)
+#pragma unroll
+                            for (int tx = 0; tx < TAPS_T; ++tx)
+#pragma unroll
+                                for (int ks = 0; ks < RB_T / 32; ++ks)
+                                    mma_i8(d, desc_hi | (a_tile + ty * a_row + (uint32_t)(tx * (RB_T / 16) + 2 * ks)),
+                                           desc_hi | (b_lo + (uint32_t)((ty * TAPS_T + tx) * (NCOLS * RB_T / 16) + 2 * ks)),
+                                           idesc, (uint32_t)(ty | tx | ks));
+                    } else {
+                        uint32_t b_j = b_lo, first = 0;
+                        for (int ty = 0; ty < taps; ++ty) {
+                            uint32_t a_j = a_tile + (uint32_t)(ty * Ws) * row16;
+                            for (int tx = 0; tx < taps; ++tx) {
+                                for (uint32_t ks = 0; ks < ksteps; ++ks) {
+                                    mma_i8(d, desc_hi | (a_j + 2 * ks), desc_hi | (b_j + 2 * ks), idesc, first);
+                                    first = 1;
+                                }
+                                a_j += row16;
+                                b_j += b_tap;
                             }
-                            a_j += row16;
-                            b_j += b_tap;
                         }
                     }
                     mma_commit(acc_full0 + 8 * slot);
@@ -346,9 +362,13 @@ cudaError_t conv_rows_launch(const void *map_a, const void *map_b, const ConvRow
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, q);
     };
-    cudaError_t e = q.n_cols == 16 ? go(conv_rows_kernel<16>)
-                    : q.n_cols == 32 ? go(conv_rows_kernel<32>)
-                    : q.n_cols == 48 ? go(conv_rows_kernel<48>) : go(conv_rows_kernel<64>);
+    cudaError_t e;
+    if (q.n_cols == 64 && q.taps == 2 && q.row_bytes == 128) e = go(conv_rows_kernel<64, 2, 128>);
+    else if (q.n_cols == 64 && q.taps == 3 && q.row_bytes == 64) e = go(conv_rows_kernel<64, 3, 64>);
+    else
+        e = q.n_cols == 16 ? go(conv_rows_kernel<16, 0, 0>)
+            : q.n_cols == 32 ? go(conv_rows_kernel<32, 0, 0>)
+            : q.n_cols == 48 ? go(conv_rows_kernel<48, 0, 0>) : go(conv_rows_kernel<64, 0, 0>);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
