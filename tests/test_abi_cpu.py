@@ -84,3 +84,39 @@ def test_bad_descriptions_are_rejected_on_the_host(lib):
     if not torch.cuda.is_available():
         status, msg = _create(pol)
         assert status == 5 and "device" in msg
+
+
+def test_further_entry_points_reject_bad_arguments_on_the_host(lib):
+    """Argument checks of the calls beside create / act happen before any device is touched."""
+    import ctypes as C
+    from paper_2211_15023_b200 import binding
+    INVALID = 1
+    buf = np.zeros(64, np.float32)
+    p = buf.ctypes.data
+    # V-trace: null array, non-positive sizes, bad clips, misaligned pointer
+    assert lib.accerl_vtrace(None, p, p, p, p, None, 2, 4, 0.99, 1.0, 1.0, p, None, None) == INVALID
+    assert lib.accerl_vtrace(p, p, p, p, p, None, 0, 4, 0.99, 1.0, 1.0, p, None, None) == INVALID
+    assert lib.accerl_vtrace(p, p, p, p, p, None, 2, 4, 0.99, -1.0, 1.0, p, None, None) == INVALID
+    assert lib.accerl_vtrace(p, p, p, p, p, None, 2, 4, 0.99, 1.0, 1.0, p + 2, None, None) == INVALID
+    assert b"vtrace" in lib.accerl_last_error()
+    # KL: null array, action count out of range
+    assert lib.accerl_policy_kl(None, p, 4, 2, p, None, None) == INVALID
+    assert lib.accerl_policy_kl(p, p, 4, 0, p, None, None) == INVALID
+    assert lib.accerl_policy_kl(p, p, 4, 2000, p, None, None) == INVALID
+    # handle-taking calls refuse a null handle
+    assert lib.accerl_policy_act_ex(None, p, p, 1, p, p, p, None, None, None) == INVALID
+    assert lib.accerl_policy_act_mixed(None, None, p, p, p, 0.5, 1, p, p, p, None, None, None, None) == INVALID
+    assert lib.accerl_policy_selftest_wait(None, 100, None) == INVALID
+    assert lib.accerl_policy_export(None, 0, None, 0, None, None, None, None) == INVALID
+    # the probe checks its shape arguments first
+    ms, cyc = C.c_float(), C.c_float()
+    assert lib.accerl_tc_probe_i8(0, 24, 1, 64, 1, 128, 0, 0, C.byref(ms), C.byref(cyc)) == INVALID
+    assert lib.accerl_tc_probe_i8(0, 256, 4, 64, 1, 128, 0, 0, C.byref(ms), C.byref(cyc)) == INVALID
+    # quantisation on the device: shapes that do not chain are refused before the device is used
+    layers = [dict(l) for l in W.config("cartpole_mlp")["layers"]]
+    params = W.fp32_parameters("cartpole_mlp")
+    calib = W.calibration_batch("cartpole_mlp", 8)
+    layers[1]["in_c"] = 63
+    with pytest.raises(binding.AccerlError) as e:
+        binding.Policy.from_fp32("f32", (4, 1, 1), layers, params, calib, 8)
+    assert e.value.status == INVALID and "layer 1" in str(e.value)
