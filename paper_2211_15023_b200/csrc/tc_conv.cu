@@ -33,7 +33,7 @@ constexpr int kMmaWarps2 = 4;            // warps 0..3 issue MMAs, the CTA's til
 constexpr int kEpiWarps2 = 16;           // warps 4..19 drain accumulators
 constexpr int kWarps2 = 4 + kEpiWarps2 + 1;  // the last warp issues the TMA loads
 constexpr int kThreads2 = 32 * kWarps2;
-constexpr int kStages2 = 3;
+constexpr int kStages2 = 4;
 constexpr int kMaxSlots2 = 16;
 
 struct __align__(8) Bars2 {
