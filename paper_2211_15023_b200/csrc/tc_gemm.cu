@@ -623,8 +623,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 nt = t - mt * p.n_tiles;
             }
             const int row0 = mt * kTileM * SUB, brow0 = nt * p.n_tile;
+            // Streamed weights: every CTA of a column of tiles reads the same weight chunks, and in
+            // lockstep they would all ask the same L2 lines at the same time.  Integer accumulation
+            // does not care about the order of K, so each row of tiles starts its K loop at a
+            // different group (the stage carries the matching A and B chunks; the issuing side never
+            // needs to know which K group a stage holds).
+            const int rot = RESIDENT_B ? 0 : mt % n_groups;
             for (int gq = 0; gq < my_groups; ++gq) {
-                const int gi = g_first + gq * g_step;
+                int gi = g_first + gq * g_step + rot;
+                if (gi >= n_groups) gi -= n_groups;
                 const int j = gi * G;
                 int sl = base_slot + gq;
                 uint32_t ph = base_phase;
