@@ -12,7 +12,8 @@
 //   sixteen 4-byte loads: 4 channels x 4 image rows), quantise four bytes at a time and write the
 //   position's 64-byte operand row.  K is ordered (channel, dy, dx) -- the order the bytes have in
 //   the frame -- and the weights are permuted to match at create, so no byte is ever transposed.
-//   The next row set's loads are in flight while the current one is converted.
+//   Each converter warp owns two fixed row sets of every step; their next loads are in flight while
+//   the current ones are converted.
 // - A tile is S whole grid rows (S * Ws <= 128 GEMM rows), so a thread of the epilogue owns the
 //   same (row, X) of every tile and decodes its output address with two multiplies.  A pipeline
 //   step is T tiles; its operand block has one grid row more than it produces (the taps reach
@@ -45,8 +46,8 @@ namespace {
 
 constexpr int kEpiWarps = 12;                       // three warpgroups
 constexpr int kMmaWarps1 = 2;                       // issuing warps (tiles of a step in turn)
-constexpr int kWarps = 24;                          // 768 threads: 80 registers each
-constexpr int kConvWarps = kWarps - kEpiWarps - kMmaWarps1;  // converter warps
+constexpr int kConvWarps = 9;                       // converter warps: two row sets of every step each
+constexpr int kWarps = kMmaWarps1 + kConvWarps + kEpiWarps;  // 23
 constexpr int kFirstExtraConv = 4 + kEpiWarps;      // converters beyond warps kMmaWarps1..3 start here
 constexpr int kThreads1 = 32 * kWarps;
 constexpr int kStages = 3;
@@ -100,7 +101,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&bars.full[s]), (uint32_t)p.sets_per_step);
+            mbar_init(smem_u32(&bars.full[s]), kConvWarps);
             mbar_init(smem_u32(&bars.empty[s]), kMmaWarps1);
         }
         for (int a = 0; a < kAccSlots; ++a) {
@@ -189,26 +190,27 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
             __syncwarp();
         }
     } else if (warp < 4 || warp >= kFirstExtraConv) {
-        static_assert(kMmaWarps1 <= 4 && kConvWarps >= 1, "roles");
         // ------------------------------------------------------------------ converters
-        // The CTA's row sets (32 grid positions each, `sets` per step) form one stream over all of its
-        // steps; warp cw takes sets cw, cw + kConvWarps, ...  Two sets are in flight per warp: while
-        // one is quantised and written, the loads of the next two travel (a single set in flight
-        // exposes the full memory latency per set).
+        // A step's operand block has at most 2 * kConvWarps row sets of 32 grid positions; warp cw
+        // owns sets cw and cw + kConvWarps of EVERY step, so a lane's two positions inside the block,
+        // their operand-row addresses and swizzles are fixed for the whole kernel and only the image
+        // and grid row behind them change from step to step.  While one set is quantised and written
+        // the loads of the warp's next two sets travel (one set in flight exposes the full memory
+        // latency per set).
+        static_assert(kMmaWarps1 <= 4 && kConvWarps >= 1, "roles");
         const int cw = warp < 4 ? warp - kMmaWarps1 : warp - kFirstExtraConv + (4 - kMmaWarps1);
         const int step_rows = (T * S + 1) * Ws;            // grid positions a step's block holds
-        const int sets = (step_rows + 31) / 32;            // row sets per step
-        const int total_sets = my_steps * sets;
-        const unsigned sets_magic = (unsigned)(((1ULL << 32) + sets - 1) / sets);  // exact far beyond total_sets
         const int W = ATARI ? 84 : p.in_w, plane = ATARI ? 84 * 84 : p.in_plane;
+        const int posA = cw * 32 + lane, posB = (cw + kConvWarps) * 32 + lane;
+        const bool vA = posA < step_rows, vB = posB < step_rows;
+        const int RlA = (int)div_ws((unsigned)posA), XA = posA - RlA * Ws;
+        const int RlB = (int)div_ws((unsigned)posB), XB = posB - RlB * Ws;
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        // loads of one position's sixteen words (zeros beyond the last image or the last set)
-        auto load = [&](uint32_t (&w)[16], int g) {
-            const int k = (int)__umulhi((unsigned)g, sets_magic), pos = (g - k * sets) * 32 + lane;
+        // loads of one position's sixteen words (zeros beyond the last image or the last step)
+        auto load = [&](uint32_t (&w)[16], int k, int Rl, int X, bool v) {
             const int step = (int)blockIdx.x + k * (int)gridDim.x;
-            const int Rl = (int)div_ws((unsigned)pos), X = pos - Rl * Ws;
             const long long R = (long long)step * (T * S) + Rl;
-            const bool in = g < total_sets && pos < step_rows && R < p.total_grid_rows;
+            const bool in = v && k < my_steps && R < p.total_grid_rows;
             const unsigned n = div_hs((unsigned)R);
             const int Y = (int)((unsigned)R - n * (unsigned)Hs);
             const uint8_t *src = p.obs + (size_t)n * 4 * plane + (size_t)(4 * Y) * W + 4 * X;
@@ -218,44 +220,36 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 for (int dy = 0; dy < 4; ++dy)
                     w[4 * c + dy] = in ? __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * plane + dy * W)) : 0u;
         };
-        bool ok = true;
-        int cur_k = -1;
-        // quantise one set and write its operand rows; the block's barrier counts one arrival per set
-        auto store = [&](const uint32_t (&w)[16], int g) {
-            const int k = (int)__umulhi((unsigned)g, sets_magic), pos = (g - k * sets) * 32 + lane;
-            const int s = k % kStages;
-            if (k != cur_k) {
-                ok = mbar_wait(empty0 + 8 * s, (uint32_t)(((k / kStages) & 1) ^ 1), abort_flag, p.status, 1);
-                ok = __all_sync(0xffffffffu, ok);
-                cur_k = k;
-                if (!ok) return;
-            }
-            uint8_t *row = stages + (size_t)s * stage_bytes + pos * 64;
-            if (pos < step_rows) {
+        // quantise one set and write its operand rows (16-byte pieces under the 64-byte swizzle)
+        auto store = [&](const uint32_t (&w)[16], uint8_t *block, int pos, bool v) {
+            if (!v) return;
+            uint8_t *row = block + pos * 64;
+            const int sw = (pos >> 1) & 3;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    *reinterpret_cast<uint4 *>(row + ((c ^ ((pos >> 1) & 3)) << 4)) =
-                        make_uint4(quantise_word<MODE>(w[4 * c], p.ingest_mul, p.ingest_add),
-                                   quantise_word<MODE>(w[4 * c + 1], p.ingest_mul, p.ingest_add),
-                                   quantise_word<MODE>(w[4 * c + 2], p.ingest_mul, p.ingest_add),
-                                   quantise_word<MODE>(w[4 * c + 3], p.ingest_mul, p.ingest_add));
-            }
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4 *>(row + ((c ^ sw) << 4)) =
+                    make_uint4(quantise_word<MODE>(w[4 * c], p.ingest_mul, p.ingest_add),
+                               quantise_word<MODE>(w[4 * c + 1], p.ingest_mul, p.ingest_add),
+                               quantise_word<MODE>(w[4 * c + 2], p.ingest_mul, p.ingest_add),
+                               quantise_word<MODE>(w[4 * c + 3], p.ingest_mul, p.ingest_add));
+        };
+        uint32_t wa[16], wb[16];
+        load(wa, 0, RlA, XA, vA);
+        load(wb, 0, RlB, XB, vB);
+        bool ok = true;
+        for (int k = 0; k < my_steps && ok; ++k) {
+            const int s = k % kStages;
+            ok = mbar_wait(empty0 + 8 * s, (uint32_t)(((k / kStages) & 1) ^ 1), abort_flag, p.status, 1);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            uint8_t *block = stages + (size_t)s * stage_bytes;
+            store(wa, block, posA, vA);
+            load(wa, k + 1, RlA, XA, vA);
+            store(wb, block, posB, vB);
+            load(wb, k + 1, RlB, XB, vB);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(full0 + 8 * s);
-        };
-        uint32_t wa[16], wb[16];
-        int g = cw;
-        load(wa, g);
-        load(wb, g + kConvWarps);
-        while (g < total_sets && ok) {
-            store(wa, g);
-            load(wa, g + 2 * kConvWarps);
-            g += kConvWarps;
-            if (g >= total_sets || !ok) break;
-            store(wb, g);
-            load(wb, g + 2 * kConvWarps);
-            g += kConvWarps;
         }
     } else {
         // ------------------------------------------------------------------ epilogue
@@ -363,6 +357,7 @@ bool conv1_plan(const accerl_layer_desc &d, int in_h, int in_w, long long max_ba
     q->n_cols = n_total;
     q->ingest_mode = ingest_mode;
     // positions a step's MMAs can touch: (T - 1) * S * Ws + 127 + Ws + 1, plus one for the count
+    if (((kMaxT * S + 1) * Ws + 31) / 32 > 2 * kConvWarps) return false;  // two row sets per converter warp and step
     q->stage_bytes = (((kMaxT - 1) * S * Ws + 128 + Ws + 1) * 64 + 1023) & ~1023;
     return true;
 }
@@ -385,7 +380,6 @@ cudaError_t conv1_launch(const void *map_b, const Conv1Params &q0, int batch, co
     while (T > 1 && (q.total_tiles + T - 1) / T < 2 * sm_count) T /= 2;
     q.tiles_per_step = T;
     q.total_steps = (q.total_tiles + T - 1) / T;
-    q.sets_per_step = ((T * q.rows_per_tile + 1) * q.grid_w + 31) / 32;
     const int grid = q.total_steps < sm_count ? q.total_steps : sm_count;
     const size_t smem = conv1_smem_bytes(q);
     auto go = [&](auto kernel) -> cudaError_t {

@@ -15,7 +15,6 @@ struct Conv1Params {
     unsigned ws_magic, hs_magic;     // ceil(2^32 / grid_w), ceil(2^32 / grid_h): division by multiply-high
     // tiling: a tile is rows_per_tile whole grid rows, a pipeline step tiles_per_step tiles
     int rows_per_tile, tiles_per_step, total_tiles, total_steps, stage_bytes;
-    int sets_per_step;               // row sets of 32 grid positions in a step's operand block
     int n_cols;                      // output channels: 16 or 32
     // input quantiser: 0 = line q = (u * mul + add) >> 24, 1 = the same with min(., 127), 2 = u >> 1
     int ingest_mode;
