@@ -8,4 +8,4 @@ raises.
 """
 from .binding import (AccerlError, Policy, act_mixed, kl, library, library_path, tc_probe_i8,  # noqa: F401
                       vtrace, FLAG_FORCE_GENERIC, FLAG_KEEP_ACTIVATIONS, FLAG_TAP_FUSED,
-                      FLAG_VALUE_HEAD, FLAG_TEST_NO_FASTDIV)
+                      FLAG_VALUE_HEAD, FLAG_TEST_NO_FASTDIV, FLAG_TEST_NO_AFFINE)

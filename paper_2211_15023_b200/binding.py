@@ -14,6 +14,7 @@ FLAG_FORCE_GENERIC = 2
 FLAG_TAP_FUSED = 4
 FLAG_VALUE_HEAD = 8
 FLAG_TEST_NO_FASTDIV = 16
+FLAG_TEST_NO_AFFINE = 32
 RELU_IN, RELU_OUT, LOGITS = 1, 2, 4
 _KINDS = {"conv": 0, "fc": 1, "maxpool": 2}
 STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "BATCH_TOO_LARGE", 4: "OOM", 5: "CUDA",

@@ -393,7 +393,8 @@ accerl_status accerl_policy_create(accerl_policy **out, int32_t in_kind, const i
         return ACCERL_ERR_INVALID_ARG;
     }
     if (flags & ~(uint32_t)(ACCERL_FLAG_KEEP_ACTIVATIONS | ACCERL_FLAG_FORCE_GENERIC | ACCERL_FLAG_TAP_FUSED |
-                            ACCERL_FLAG_VALUE_HEAD | ACCERL_FLAG_TEST_NO_FASTDIV)) {
+                            ACCERL_FLAG_VALUE_HEAD | ACCERL_FLAG_TEST_NO_FASTDIV |
+                            ACCERL_FLAG_TEST_NO_AFFINE)) {
         set_error("create: unknown flag bits 0x%x", flags);
         return ACCERL_ERR_INVALID_ARG;
     }

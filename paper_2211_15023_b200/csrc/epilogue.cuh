@@ -79,19 +79,25 @@ __device__ __forceinline__ void requant16(const int (&acc)[16], const float (&ks
     for (int g = 0; g < 4; ++g) w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
 }
 
+// max(code, 0) on four signed bytes: a byte permute in its sign-replicating mode gives 0xff for
+// every negative byte, and those bytes are cleared
+__device__ __forceinline__ uint32_t relu_bytes(uint32_t w)
+{
+    uint32_t neg;
+    asm("prmt.b32 %0, %1, %1, 0xba98;" : "=r"(neg) : "r"(w));
+    return w & ~neg;
+}
+
 // One requantised code by the three-step division: t = y * r, e = y - s * t (exact in one fma),
 // d = t + e * r.  With r = fl(1 / s) this is the classical correctly rounded quotient except for
 // rare operand patterns, so it is only used for scales for which fastdiv_code() has been compared
 // with exact_code() over every fp32 value y can take (see verify_fastdiv in tc_plan.cu).  ReLU
-// is applied to the quotient, which has the sign of y; the saturating pack does the clamp.
-template <bool RELU>
+// is applied to the code, which has the sign of y; the saturating pack does the clamp.
 __device__ __forceinline__ int fastdiv_rint(float y, float s, float r)
 {
     const float t = __fmul_rn(y, r);
     const float e = __fmaf_rn(-s, t, y);
-    float d = __fmaf_rn(e, r, t);
-    if (RELU) d = fmaxf(d, 0.f);  // the quotient has the sign of y
-    return __float2int_rn(d);
+    return __float2int_rn(__fmaf_rn(e, r, t));
 }
 
 // the defining expression, for one element: clamp(rintf(max?(y) / s), -128, 127)
@@ -104,12 +110,13 @@ __device__ __forceinline__ int exact_code(float y, float s, bool relu)
 template <bool RELU>
 __device__ __forceinline__ int fastdiv_code(float y, float s, float r)
 {
-    return min(max(fastdiv_rint<RELU>(y, s, r), -128), 127);  // what the saturating pack does
+    const int q = min(max(fastdiv_rint(y, s, r), -128), 127);  // what the saturating pack does
+    return RELU ? max(q, 0) : q;                               // and relu_bytes()
 }
 
 // Sixteen codes by the three-step division, two elements per instruction: the packed fp32
 // operations of sm_100 round each half exactly as their scalar forms do, so the codes are those
-// of fastdiv_rint(); they only take half the issue slots.
+// of fastdiv_code(); they only take half the issue slots.
 template <bool RELU>
 __device__ __forceinline__ void requant16_fastdiv(const int (&acc)[16], const float (&ks)[16],
                                                   const float (&bs)[16], float s_out,
@@ -123,16 +130,47 @@ __device__ __forceinline__ void requant16_fastdiv(const int (&acc)[16], const fl
         const float2 y = __ffma2_rn(a, make_float2(ks[i], ks[i + 1]), make_float2(bs[i], bs[i + 1]));
         const float2 t = __fmul2_rn(y, r2);
         const float2 e = __ffma2_rn(ns2, t, y);
-        float2 d = __ffma2_rn(e, r2, t);
-        if (RELU) {  // the quotient has the sign of y
-            d.x = fmaxf(d.x, 0.f);
-            d.y = fmaxf(d.y, 0.f);
-        }
+        const float2 d = __ffma2_rn(e, r2, t);
         q[i] = __float2int_rn(d.x);
         q[i + 1] = __float2int_rn(d.y);
     }
 #pragma unroll
-    for (int g = 0; g < 4; ++g) w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
+    for (int g = 0; g < 4; ++g) {
+        w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
+        if (RELU) w[g] = relu_bytes(w[g]);
+    }
+}
+
+// One code by a single fma: q = clamp(rint(fmaf((float)acc, k2, b2))), ReLU on the code.  The
+// requantiser is a non-decreasing step function of the INTEGER accumulator, and so is this one
+// (k2 > 0); for every output channel the pair (k2, b2) near (k / s_out, b / s_out) is searched at
+// create until the two functions agree on every accumulator between the two points where both
+// saturate, which makes them equal on all of int32 (fit_affine_requant in requant_fit.cu).
+template <bool RELU>
+__device__ __forceinline__ int affine_code(int acc, float k2, float b2)
+{
+    const int q = min(max(__float2int_rn(__fmaf_rn(__int2float_rn(acc), k2, b2)), -128), 127);
+    return RELU ? max(q, 0) : q;
+}
+
+// sixteen codes by the single fma, two elements per instruction
+template <bool RELU>
+__device__ __forceinline__ void requant16_affine(const int (&acc)[16], const float (&k2)[16],
+                                                 const float (&b2)[16], uint32_t (&w)[4])
+{
+    int q[16];
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        const float2 a = make_float2(__int2float_rn(acc[i]), __int2float_rn(acc[i + 1]));
+        const float2 t = __ffma2_rn(a, make_float2(k2[i], k2[i + 1]), make_float2(b2[i], b2[i + 1]));
+        q[i] = __float2int_rn(t.x);
+        q[i + 1] = __float2int_rn(t.y);
+    }
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        w[g] = pack4_sat_s8(q[4 * g], q[4 * g + 1], q[4 * g + 2], q[4 * g + 3]);
+        if (RELU) w[g] = relu_bytes(w[g]);
+    }
 }
 
 // Four frame bytes (byte `dx` of the words p0..p3, one per channel plane) -> four int8 codes in one

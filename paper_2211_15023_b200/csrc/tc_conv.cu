@@ -49,7 +49,7 @@ struct __align__(8) Bars2 {
 // TAPS_T / RB_T: taps per side and bytes of an operand row as compile-time constants (0 = taken from
 // the parameters); with them the issue loop of a tile is straight-line code, and the issuing warps'
 // instruction count is what bounds how fast tiles start.
-template <int NCOLS, int TAPS_T, int RB_T>
+template <int NCOLS, int TAPS_T, int RB_T, bool AFFINE>
 __global__ void __launch_bounds__(kThreads2, 1)
 conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const __grid_constant__ ConvRowsParams p)
@@ -239,8 +239,13 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             bs[e] = p.bs[32 * hh + 16 * h + e];
                         }
                         uint32_t wv[4];
-                        if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
-                        else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                        if (AFFINE) {
+                            if (p.relu) requant16_affine<true>(acc[h], ks, bs, wv);
+                            else requant16_affine<false>(acc[h], ks, bs, wv);
+                        } else {
+                            if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                            else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                        }
                         if (valid) *reinterpret_cast<uint4 *>(dst + 32 * hh + 16 * h) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
                     }
                 }
@@ -363,12 +368,18 @@ cudaError_t conv_rows_launch(const void *map_a, const void *map_b, const ConvRow
         return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, q);
     };
     cudaError_t e;
-    if (q.n_cols == 64 && q.taps == 2 && q.row_bytes == 128) e = go(conv_rows_kernel<64, 2, 128>);
-    else if (q.n_cols == 64 && q.taps == 3 && q.row_bytes == 64) e = go(conv_rows_kernel<64, 3, 64>);
+    // (the requantiser is a template parameter, not a branch: both epilogues in one kernel cost time)
+    if (q.n_cols == 64 && q.taps == 2 && q.row_bytes == 128)
+        e = q.affine ? go(conv_rows_kernel<64, 2, 128, true>) : go(conv_rows_kernel<64, 2, 128, false>);
+    else if (q.n_cols == 64 && q.taps == 3 && q.row_bytes == 64)
+        e = q.affine ? go(conv_rows_kernel<64, 3, 64, true>) : go(conv_rows_kernel<64, 3, 64, false>);
     else
-        e = q.n_cols == 16 ? go(conv_rows_kernel<16, 0, 0>)
-            : q.n_cols == 32 ? go(conv_rows_kernel<32, 0, 0>)
-            : q.n_cols == 48 ? go(conv_rows_kernel<48, 0, 0>) : go(conv_rows_kernel<64, 0, 0>);
+        e = q.affine ? (q.n_cols == 16 ? go(conv_rows_kernel<16, 0, 0, true>)
+                        : q.n_cols == 32 ? go(conv_rows_kernel<32, 0, 0, true>)
+                        : q.n_cols == 48 ? go(conv_rows_kernel<48, 0, 0, true>) : go(conv_rows_kernel<64, 0, 0, true>))
+                     : (q.n_cols == 16 ? go(conv_rows_kernel<16, 0, 0, false>)
+                        : q.n_cols == 32 ? go(conv_rows_kernel<32, 0, 0, false>)
+                        : q.n_cols == 48 ? go(conv_rows_kernel<48, 0, 0, false>) : go(conv_rows_kernel<64, 0, 0, false>));
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

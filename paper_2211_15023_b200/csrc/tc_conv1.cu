@@ -85,7 +85,7 @@ __device__ __forceinline__ uint32_t quantise_word(uint32_t w, uint32_t mul, uint
 
 // ATARI: the frame is 84 x 84 (a 21 x 21 grid, tiles of six grid rows); the divisions, strides and
 // load offsets are then compile-time constants, which takes a third off the converters' instructions.
-template <int NCOLS, int MODE, bool ATARI>
+template <int NCOLS, int MODE, bool ATARI, bool AFFINE>
 __global__ void __launch_bounds__(kThreads1, 1)
 conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_constant__ Conv1Params p)
 {
@@ -298,8 +298,13 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                         bs[e] = p.bs[16 * h + e];
                     }
                     uint32_t wv[4];
-                    if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
-                    else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                    if (AFFINE) {
+                        if (p.relu) requant16_affine<true>(acc[h], ks, bs, wv);
+                        else requant16_affine<false>(acc[h], ks, bs, wv);
+                    } else {
+                        if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                        else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
+                    }
                     if (valid) *reinterpret_cast<uint4 *>(dst + 16 * h) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
                 }
             }
@@ -398,11 +403,16 @@ cudaError_t conv1_launch(const void *map_b, const Conv1Params &q0, int batch, co
         return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_b, q);
     };
     const bool atari = q.in_w == 84 && q.in_plane == 84 * 84;
+    // (the requantiser is a template parameter, not a branch: with both epilogues in one kernel the
+    // layer measured 4 to 7 us slower)
     auto pick = [&](auto ncols, auto is_atari) -> cudaError_t {
         constexpr int N = decltype(ncols)::value;
         constexpr bool A = decltype(is_atari)::value;
-        return q.ingest_mode == 2 ? go(conv1_frames_kernel<N, 2, A>)
-               : q.ingest_mode == 1 ? go(conv1_frames_kernel<N, 1, A>) : go(conv1_frames_kernel<N, 0, A>);
+        if (q.affine)
+            return q.ingest_mode == 2 ? go(conv1_frames_kernel<N, 2, A, true>)
+                   : q.ingest_mode == 1 ? go(conv1_frames_kernel<N, 1, A, true>) : go(conv1_frames_kernel<N, 0, A, true>);
+        return q.ingest_mode == 2 ? go(conv1_frames_kernel<N, 2, A, false>)
+               : q.ingest_mode == 1 ? go(conv1_frames_kernel<N, 1, A, false>) : go(conv1_frames_kernel<N, 0, A, false>);
     };
     cudaError_t e;
     if (q.n_cols == 32)

@@ -25,6 +25,7 @@ struct Conv1Params {
     int out_h, out_w, out_s2d_log2, out_rows_per_image, out_grid_w, out_pitch, n_total;
     float s_out, inv_s_out;
     int relu;
+    int affine;                      // 1: ks / bs are the single-fma constants (k2, b2)
     float ks[32], bs[32];            // s_in * s_w[c] and bias per output channel
     int *status;
 };

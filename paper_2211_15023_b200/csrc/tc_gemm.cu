@@ -31,6 +31,7 @@
 #include "tc_ptx.cuh"
 
 #include <algorithm>
+#include <type_traits>
 
 namespace accerl {
 
@@ -73,7 +74,7 @@ struct EpiCtx {
     uint8_t *staging;  // kStagingBytes per epilogue warp when the layer stores through shared memory
 };
 
-enum { kEpiFastDiv = 0, kEpiTieCheck = 1, kEpiLogits = 2 };
+enum { kEpiFastDiv = 0, kEpiTieCheck = 1, kEpiLogits = 2, kEpiAffine = 3 };
 constexpr int kStagingBytes = 32 * 128;  // 32 rows of 128 output bytes
 
 // byte offset of 16-byte piece `ch` of row `row` in a warp's staging tile; the XOR spreads a
@@ -84,10 +85,7 @@ __device__ __forceinline__ uint4 relu_codes(uint4 v)
 {
     uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-    for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
-        const uint32_t neg = w[g] & 0x80808080u;
-        w[g] &= ~(neg | (neg - (neg >> 7)));
-    }
+    for (int g = 0; g < 4; ++g) w[g] = relu_bytes(w[g]);
     return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
@@ -242,7 +240,8 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                     continue;
                 }
                 uint32_t w[4];
-                if (MODE == kEpiFastDiv) requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+                if (MODE == kEpiAffine) requant16_affine<RELU>(acc, ks, bs, w);
+                else if (MODE == kEpiFastDiv) requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
                 else requant16(acc, ks, bs, RELU, s_out, inv_s_out, w);
                 const uint4 plain = make_uint4(w[0], w[1], w[2], w[3]);
                 if (STAGED) {
@@ -252,10 +251,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                     if (p.out_relu | p.out2_relu) {
                         uint32_t wr[4];
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {  // max(code, 0) on four signed bytes
-                            const uint32_t neg = w[g] & 0x80808080u;
-                            wr[g] = w[g] & ~(neg | (neg - (neg >> 7)));
-                        }
+                        for (int g = 0; g < 4; ++g) wr[g] = relu_bytes(w[g]);
                         relu = make_uint4(wr[0], wr[1], wr[2], wr[3]);
                     }
                     if (valid && c0 < n_store) {
@@ -291,7 +287,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
 // on every other tile (two tiles are drained at a time, one per accumulator stage); inside a pair a
 // warp produces two of the row's four (pooled pixel, 16-channel piece) items, each from the
 // accumulators of pixels 2j .. 2j+2.
-template <bool RELU>
+template <bool RELU, bool AFFINE>
 __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
 {
     const int q = warp & 3, wg = (warp - kProdWarps - kMmaWarps) >> 2;
@@ -350,7 +346,8 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
                 bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
             }
             uint32_t w[4];
-            requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+            if (AFFINE) requant16_affine<RELU>(acc, ks, bs, w);
+            else requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
             if (row_ok && X * (4 / hpc) + ox < p.px_w)
                 *reinterpret_cast<uint4 *>(dst_row + ox * p.out_pitch + 16 * half) = make_uint4(w[0], w[1], w[2], w[3]);
         }
@@ -409,7 +406,7 @@ __device__ __forceinline__ void convert_tile(const TcGemmParams &p, const uint8_
 // FUSE is the first conv with the input stage inside (TcGemmParams::fuse_ingest).
 // PXK is the kernel for rows of several output pixels; it is kept apart so that its epilogue
 // variants do not weigh on the register allocation of the others.
-template <bool RESIDENT_B, bool EXTRAS, bool PXK, bool FUSE>
+template <bool RESIDENT_B, bool EXTRAS, bool PXK, bool FUSE, bool AFFINE>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcGemmParams p)
@@ -795,17 +792,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         c.staging = stages + (size_t)n_stages * stage_bytes;
         // outputs may reuse buffers that the previous launch still reads
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        if constexpr (PXK) {  // multi-pixel rows: only built for the verified division
+        // (the requantiser is a template parameter of the kernel, not a branch: with both epilogues in
+        // one kernel the layers measured slower)
+        constexpr int kDivFree = AFFINE ? kEpiAffine : kEpiFastDiv;
+        if constexpr (PXK) {  // multi-pixel rows: only built for the verified requantisers
             if (p.hpool) {
-                if (p.relu_out) epilogue_hpool<true>(p, c, warp, lane);
-                else epilogue_hpool<false>(p, c, warp, lane);
+                if (p.relu_out) epilogue_hpool<true, AFFINE>(p, c, warp, lane);
+                else epilogue_hpool<false, AFFINE>(p, c, warp, lane);
             } else if (p.staged) {
-                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, true, KS>(p, c, warp, lane);
-                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, true, KS>(p, c, warp, lane);
+                if (p.relu_out) epilogue_role<EXTRAS, kDivFree, true, true, true, KS>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kDivFree, false, true, true, KS>(p, c, warp, lane);
             } else {
-                if (p.relu_out) epilogue_role<EXTRAS, kEpiFastDiv, true, true, false, KS>(p, c, warp, lane);
-                else epilogue_role<EXTRAS, kEpiFastDiv, false, true, false, KS>(p, c, warp, lane);
+                if (p.relu_out) epilogue_role<EXTRAS, kDivFree, true, true, false, KS>(p, c, warp, lane);
+                else epilogue_role<EXTRAS, kDivFree, false, true, false, KS>(p, c, warp, lane);
             }
+        } else if constexpr (AFFINE) {
+            if (p.relu_out) epilogue_role<EXTRAS, kEpiAffine, true, false, false, KS>(p, c, warp, lane);
+            else epilogue_role<EXTRAS, kEpiAffine, false, false, false, KS>(p, c, warp, lane);
         } else {
             if (p.logits_mode) epilogue_role<false, kEpiLogits, false, false, false, KS>(p, c, warp, lane);
             else if (p.fast_div) {
@@ -974,20 +977,23 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
         return cudaLaunchKernelEx(&cfg, kernel, *(const CUtensorMap *)map_a, *(const CUtensorMap *)map_b, q);
     };
     cudaError_t e;
-    if (p.px_per_row) {
-        if (!resident_b || !p.fast_div || p.logits_mode) return cudaErrorInvalidValue;
-        e = extras ? go(tc_gemm_kernel<true, true, true, false>) : go(tc_gemm_kernel<true, false, true, false>);
-    } else {
+    if (p.affine && (!p.fast_div || p.logits_mode)) return cudaErrorInvalidValue;
+    auto pick = [&](auto affine) -> cudaError_t {
+        constexpr bool A = decltype(affine)::value;
+        if (p.px_per_row) {
+            if (!resident_b || !p.fast_div || p.logits_mode) return cudaErrorInvalidValue;
+            return extras ? go(tc_gemm_kernel<true, true, true, false, A>) : go(tc_gemm_kernel<true, false, true, false, A>);
+        }
         if (p.fuse_ingest) {
             if (!resident_b || extras || !p.shifted || p.n_stages != p.n_mma) return cudaErrorInvalidValue;
-            e = go(tc_gemm_kernel<true, false, false, true>);
-        } else {
-            e = resident_b ? (extras ? go(tc_gemm_kernel<true, true, false, false>)
-                                     : go(tc_gemm_kernel<true, false, false, false>))
-                           : (extras ? go(tc_gemm_kernel<false, true, false, false>)
-                                     : go(tc_gemm_kernel<false, false, false, false>));
+            return go(tc_gemm_kernel<true, false, false, true, A>);
         }
-    }
+        return resident_b ? (extras ? go(tc_gemm_kernel<true, true, false, false, A>)
+                                    : go(tc_gemm_kernel<true, false, false, false, A>))
+                          : (extras ? go(tc_gemm_kernel<false, true, false, false, A>)
+                                    : go(tc_gemm_kernel<false, false, false, false, A>));
+    };
+    e = p.affine ? pick(std::true_type()) : pick(std::false_type());
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

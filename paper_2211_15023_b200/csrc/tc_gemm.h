@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "accerl.h"
 
 namespace accerl {
@@ -68,6 +70,7 @@ struct TcGemmParams {
     const float *kscale, *bias;
     float s_out, inv_s_out;
     int fast_div;  // 1: the three-step division has been verified for this s_out (epilogue.cuh)
+    int affine;    // 1: kscale / bias hold the verified single-fma constants (requant_fit.cu)
     int relu_out;
     int split_cols;  // 1: the four epilogue warpgroups share a tile (a quarter of the columns each)
     // 1: rows leave through a shared-memory tile per warp, eight lanes per row (needs n_tile = 128,
@@ -106,6 +109,8 @@ cudaError_t launch_ingest_u8_s2d(const uint8_t *obs, const int8_t *lut, int8_t *
 // exhaustive check of the three-step division against the IEEE divide for one output scale
 accerl_status verify_fastdiv(float s_out, float inv_s_out, bool relu, float y_max, bool *ok);
 accerl_status choose_fastdiv(float s_out, bool relu, float y_max, bool allow, float *inv_s_out, int *fast_div);
+accerl_status fit_affine_requant(const float *k, const float *b, int n, float s_out, bool relu,
+                                 std::vector<float> *k2, std::vector<float> *b2, bool *ok);
 bool fit_ingest_line(const int8_t *lut, uint32_t *mul, uint32_t *add);
 bool fit_ingest_float_line(const int8_t *lut, uint32_t mul, uint32_t add, uint32_t *a_bits, uint32_t *c1_bits);
 

@@ -735,6 +735,29 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                                 !(p->flags & ACCERL_FLAG_TEST_NO_FASTDIV), &g.inv_s_out, &g.fast_div);
             if (st != ACCERL_OK) return st;
         }
+        // the single-fma requantiser where every channel has verified constants
+        if (!logits && g.fast_div && !(p->flags & ACCERL_FLAG_TEST_NO_AFFINE)) {
+            const bool repeated = role[i] == TCFIRST || P;  // columns = (pixel of the row, channel)
+            std::vector<float> kh(n_total, 0.f), bh(n_total, 0.f), k2, b2;
+            for (int j = 0; j < n_total; ++j) {
+                const int oc = repeated ? j % d.out_c : j;
+                if (oc >= d.out_c) continue;
+                volatile float k = d.s_in * d.s_w[oc];
+                kh[j] = k;
+                bh[j] = d.bias[oc];
+            }
+            bool ok = false;
+            st = fit_affine_requant(kh.data(), bh.data(), n_total, g.s_out, g.relu_out != 0, &k2, &b2, &ok);
+            if (st != ACCERL_OK) return st;
+            if (ok) {
+                void *kd = nullptr, *bd = nullptr;
+                if ((st = upload_bytes(p, k2.data(), k2.size() * 4, &kd)) != ACCERL_OK) return st;
+                if ((st = upload_bytes(p, b2.data(), b2.size() * 4, &bd)) != ACCERL_OK) return st;
+                g.kscale = (const float *)kd;
+                g.bias = (const float *)bd;
+                g.affine = 1;
+            }
+        }
         g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first) || hp_out) ? 1 : 0;
         if (role[i] == TCPX && !g.fast_div) {  // multi-pixel rows need the verified division
             p->plan_note = "tensor-core plan not used: the division-free requantiser could not be verified for the "
@@ -783,7 +806,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         s.kind = Step::TC_GEMM;
         s.tc = (int)p->tc_steps.size() - 1;
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
-        if (g.fast_div) s.kernel += "[3-step divide verified]";
+        if (g.fast_div) s.kernel += g.affine ? "[single-fma requantiser verified]" : "[3-step divide verified]";
         if (g.hpool) s.kernel += "[pooled along x on the accumulators]";
         steps.push_back(s);
     }

@@ -438,6 +438,31 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                                               allow_fastdiv, &g.inv_s_out, &g.fast_div);
             if (vs != ACCERL_OK) return vs;
         }
+        // the single-fma requantiser where every channel has verified constants
+        std::vector<float> k_use(n_total, 0.f), b_use(n_total, 0.f);
+        for (int c = 0; c < d.out_c; ++c) {
+            volatile float k = d.s_in * d.s_w[c];  // one fp32 rounding, never contracted
+            k_use[c] = k;
+            b_use[c] = d.bias[c];
+        }
+        if (!logits && g.fast_div && !(p->flags & ACCERL_FLAG_TEST_NO_AFFINE)) {
+            bool ok = false;
+            std::vector<float> k2, b2;
+            accerl_status vs = fit_affine_requant(k_use.data(), b_use.data(), n_total, g.s_out, g.relu_out != 0,
+                                                  &k2, &b2, &ok);
+            if (vs != ACCERL_OK) return vs;
+            if (ok) {
+                void *kd = nullptr, *bd = nullptr;
+                if ((vs = upload_bytes(p, k2.data(), k2.size() * 4, &kd)) != ACCERL_OK) return vs;
+                if ((vs = upload_bytes(p, b2.data(), b2.size() * 4, &bd)) != ACCERL_OK) return vs;
+                g.kscale = (const float *)kd;
+                g.bias = (const float *)bd;
+                g.affine = 1;
+                k_use = k2;
+                b_use = b2;
+            }
+        }
+        const char *requant_note = g.affine ? "[single-fma requantiser verified]" : "[3-step divide verified]";
         g.split_cols = g.n_tile >= 128 ? 1 : 0;  // 128 / 256 columns: 32 / 64 per warpgroup
         g.out = L.out_buf >= 0 ? p->bufs[L.out_buf].ptr : nullptr;
         g.logits_mode = logits ? 1 : 0;
@@ -498,11 +523,11 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 c1.s_out = g.s_out;
                 c1.inv_s_out = g.inv_s_out;
                 c1.relu = g.relu_out;
+                c1.affine = g.affine;
                 c1.status = p->status_word;
                 for (int c = 0; c < n_total; ++c) {
-                    volatile float k = d.s_in * d.s_w[c];  // one fp32 rounding, never contracted
-                    c1.ks[c] = k;
-                    c1.bs[c] = d.bias[c];
+                    c1.ks[c] = k_use[c];
+                    c1.bs[c] = b_use[c];
                 }
                 // weights [tap][channel][64 bytes], K ordered (c, dy, dx) as the bytes lie in the frame
                 std::vector<int8_t> w1((size_t)4 * n_total * 64, 0);
@@ -523,7 +548,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 Step s;
                 s.kind = Step::CONV1_FRAMES;
                 s.layer = i;
-                s.kernel = "conv1_frames_kernel[3-step divide verified][frames quantised inside]";
+                s.kernel = std::string("conv1_frames_kernel") + requant_note + "[frames quantised inside]";
                 s.covers = "ingest+layer 0";
                 steps.clear();
                 p->tap_missing[0] = 1;  // no quantised input tensor exists
@@ -552,11 +577,11 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 c2.s_out = g.s_out;
                 c2.inv_s_out = g.inv_s_out;
                 c2.relu = g.relu_out;
+                c2.affine = g.affine;
                 c2.status = p->status_word;
                 for (int c = 0; c < d.out_c; ++c) {
-                    volatile float k = d.s_in * d.s_w[c];  // one fp32 rounding, never contracted
-                    c2.ks[c] = k;
-                    c2.bs[c] = d.bias[c];
+                    c2.ks[c] = k_use[c];
+                    c2.bs[c] = b_use[c];
                 }
                 void *w2_dev = nullptr;
                 accerl_status st2 = upload_bytes(p, packed.data(), packed.size(), &w2_dev);
@@ -572,7 +597,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
                 s.kind = Step::CONV_ROWS;
                 s.layer = i;
                 s.tc = (int)p->conv_rows.size() - 1;
-                s.kernel = "conv_rows_kernel[3-step divide verified]";
+                s.kernel = std::string("conv_rows_kernel") + requant_note;
                 s.covers = "layer " + std::to_string(i);
                 steps.push_back(s);
                 continue;
@@ -606,7 +631,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         s.layer = i;
         s.tc = (int)p->tc_steps.size() - 1;
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
-        if (g.fast_div) s.kernel += "[3-step divide verified]";
+        if (g.fast_div) s.kernel += requant_note;
         s.covers = "layer " + std::to_string(i);
         if (g.fuse_ingest) {  // takes the place of the ingest launch
             s.kernel += "[frames quantised inside]";

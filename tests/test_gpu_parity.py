@@ -424,13 +424,15 @@ def test_exact_ties_on_the_tensor_core_path():
         s_prev = l["s_out"]
     assert ties > 200, ties
     ref = oracle.forward(pol, obs, u)
-    g = P.Policy(pol, b, flags=1)
-    assert "tc_gemm" in g.info()["plan"]
-    # power-of-two scales are the easy case of the three-step division: it must have been verified
-    assert "3-step divide verified" in g.info()["plan"]
-    out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
-    compare(ref, *out, taps=g.read_activation)
-    g.close()
+    # power-of-two scales are the easy case of both division-free requantisers: the single fma is
+    # exact, and so is the three-step division it replaces
+    for flags, note in ((1, "single-fma requantiser verified"), (1 | P.FLAG_TEST_NO_AFFINE, "3-step divide verified")):
+        g = P.Policy(pol, b, flags=flags)
+        assert "tc_gemm" in g.info()["plan"]
+        assert note in g.info()["plan"], g.info()["plan"]
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        compare(ref, *out, taps=g.read_activation)
+        g.close()
 
 
 def test_abi_rejects_bad_calls_without_launching():
@@ -465,7 +467,7 @@ def test_policies_whose_output_scales_fail_the_division_check(name, b):
     for flags in (P.FLAG_TEST_NO_FASTDIV, P.FLAG_TEST_NO_FASTDIV | 5):
         g = P.Policy(pol, b, flags=flags)
         plan = g.info()["plan"]
-        assert "3-step divide verified" not in plan, plan
+        assert "3-step divide verified" not in plan and "single-fma" not in plan, plan
         if name == "impala_resnet_b16384":
             assert "note: tensor-core plan not used" in plan and "conv_dp4a_kernel" in plan, plan
         else:
@@ -474,3 +476,30 @@ def test_policies_whose_output_scales_fail_the_division_check(name, b):
         g.check()
         compare(ref, *out, taps=g.read_activation if flags & 1 else None)
         g.close()
+
+
+@pytest.mark.parametrize("name,b", [("nature_cnn_b8192", 200), ("student_cnn_b8192", 141), ("impala_resnet_b16384", 9),
+                                    ("lunarlander_mlp", 300)])
+def test_single_fma_requantiser_and_the_division_it_replaces_give_the_same_bits(name, b):
+    """At create every requantising layer of a tensor-core plan searches, per output channel, the
+    constants of a one-fma requantiser that equals the defining expression on every int32
+    accumulator.  The workloads' conv layers find them (the plan says so); with the test flag the
+    search is skipped and the verified three-step division runs instead.  Both against the oracle,
+    tensor by tensor."""
+    import paper_2211_15023_b200 as P
+    pol = calibrated(name, 64)
+    obs, u = W.observations(name, b), W.uniforms(name, b)
+    ref = oracle.forward(pol, obs, u)
+    for flags in (P.FLAG_KEEP_ACTIVATIONS | P.FLAG_TAP_FUSED, P.FLAG_KEEP_ACTIVATIONS | P.FLAG_TAP_FUSED | P.FLAG_TEST_NO_AFFINE, 0):
+        g = P.Policy(pol, b, flags=flags)
+        plan = g.info()["plan"]
+        if "tc_gemm" in plan or "conv1_frames" in plan:
+            if flags & P.FLAG_TEST_NO_AFFINE:
+                assert "single-fma" not in plan and "3-step divide verified" in plan, plan
+            else:  # the conv layers find their constants; a wide fc layer may have a channel without
+                assert plan.count("single-fma requantiser verified") >= 2, plan
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        g.check()
+        compare(ref, *out, taps=g.read_activation if flags & 1 else None)
+        g.close()
+
