@@ -206,19 +206,21 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
         const int RlA = (int)div_ws((unsigned)posA), XA = posA - RlA * Ws;
         const int RlB = (int)div_ws((unsigned)posB), XB = posB - RlB * Ws;
         asm volatile("griddepcontrol.wait;" ::: "memory");
-        // loads of one position's sixteen words (zeros beyond the last image or the last step)
+        // loads of one position's sixteen words; never predicated: a position beyond the last image or
+        // the last step reads the first image's bytes instead (its row is no output), which takes the
+        // sixteen selects out of the loop (86 against 89.5 us for the layer)
         auto load = [&](uint32_t (&w)[16], int k, int Rl, int X, bool v) {
             const int step = (int)blockIdx.x + k * (int)gridDim.x;
             const long long R = (long long)step * (T * S) + Rl;
             const bool in = v && k < my_steps && R < p.total_grid_rows;
             const unsigned n = div_hs((unsigned)R);
             const int Y = (int)((unsigned)R - n * (unsigned)Hs);
-            const uint8_t *src = p.obs + (size_t)n * 4 * plane + (size_t)(4 * Y) * W + 4 * X;
+            const uint8_t *src = p.obs + (in ? (size_t)n * 4 * plane + (size_t)(4 * Y) * W + 4 * X : (size_t)0);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int dy = 0; dy < 4; ++dy)
-                    w[4 * c + dy] = in ? __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * plane + dy * W)) : 0u;
+                    w[4 * c + dy] = __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * plane + dy * W));
         };
         // quantise one set and write its operand rows (16-byte pieces under the 64-byte swizzle)
         auto store = [&](const uint32_t (&w)[16], uint8_t *block, int pos, bool v) {
