@@ -26,7 +26,7 @@
 //   113 against 94 us for the layer).
 //
 // Roles: warps 0..kMmaWarps1-1 issue MMAs (warp 0 owns tensor memory), the rest of warps 0..3 and
-// warps kFirstExtraConv.. convert,
+// warps kFirstExtraConv..kWarps-2 convert, the last warp prefetches frames into L2,
 // warps 4..4+kEpiWarps-1 drain accumulators (warp w reads lane quarter w % 4).  Rings: kStages
 // operand blocks (full / empty barriers), kAccSlots accumulators of 32 columns (one per tile).
 // Every wait is bounded; a wait that gives up sets the status word and all roles leave.
@@ -47,8 +47,10 @@ namespace {
 constexpr int kEpiWarps = 12;                       // three warpgroups
 constexpr int kMmaWarps1 = 2;                       // issuing warps (tiles of a step in turn)
 constexpr int kConvWarps = 9;                       // converter warps: two row sets of every step each
-constexpr int kWarps = kMmaWarps1 + kConvWarps + kEpiWarps;  // 23
+constexpr int kWarps = kMmaWarps1 + kConvWarps + kEpiWarps + 1;  // 24: the last one prefetches
 constexpr int kFirstExtraConv = 4 + kEpiWarps;      // converters beyond warps kMmaWarps1..3 start here
+constexpr int kPrefetchWarp = kWarps - 1;
+constexpr int kPrefetchAhead = 3;                   // steps between a block being full and the prefetched one
 constexpr int kThreads1 = 32 * kWarps;
 constexpr int kStages = 3;
 constexpr int kAccSlots = 16;  // x 32 columns = all 512 columns of tensor memory
@@ -60,6 +62,7 @@ struct __align__(8) Bars1 {
     uint64_t b_ready;
     uint32_t tmem_base;
     int abort_flag;
+    int conv_progress;  // steps the first converter warp has finished: paces the prefetch warp
 };
 
 // four frame bytes -> four codes by the fixed-point line q = min((u * mul + add) >> 24, 127)
@@ -110,6 +113,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
         }
         mbar_init(smem_u32(&bars.b_ready), 1);
         bars.abort_flag = 0;
+        bars.conv_progress = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -189,6 +193,45 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
             if (ok && elect_one()) mma_commit(empty0 + 8 * s);  // the block is free when these MMAs retire
             __syncwarp();
         }
+    } else if (warp == kPrefetchWarp) {
+        // ------------------------------------------------------------------ L2 prefetch
+        // A converter warp has its loads in flight for one step only (two row sets fill its
+        // registers), less than the memory latency under load.  This warp asks for the frame bytes of
+        // the step kPrefetchAhead after the one just converted to be brought into L2, so that the
+        // converters' loads find them there: whole image rows, up to eight runs of grid rows x four
+        // planes per step, one bulk prefetch per lane.  (Issuing them from a converter warp made that
+        // warp the slowest: the twelve-odd bulk operations take it about 900 cycles a step.)
+        const int W = ATARI ? 84 : p.in_w, plane = ATARI ? 84 * 84 : p.in_plane;
+        auto prefetch = [&](int k) {
+            if (k >= my_steps) return;
+            const int step = (int)blockIdx.x + k * (int)gridDim.x;
+            const long long R0 = (long long)step * (T * S);
+            const unsigned n0 = div_hs((unsigned)R0);
+            const int seg = lane >> 2, c = lane & 3;  // run `seg` of the step lies in image n0 + seg
+            const long long Ra = seg == 0 ? R0 : (long long)(n0 + seg) * Hs;
+            long long Rb = (long long)(n0 + seg + 1) * Hs;
+            Rb = Rb < R0 + T * S + 1 ? Rb : R0 + T * S + 1;
+            Rb = Rb < p.total_grid_rows ? Rb : p.total_grid_rows;
+            if (Ra >= Rb) return;
+            const int Y = (int)(Ra - (long long)(n0 + seg) * Hs);
+            const uint8_t *src = p.obs + ((size_t)(n0 + seg) * 4 + c) * plane + (size_t)(4 * Y) * W;
+            const uint32_t bytes = (uint32_t)(Rb - Ra) * (uint32_t)(4 * W);  // 16-byte multiples: W % 4 == 0
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+        };
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        for (int k = 1; k < kPrefetchAhead; ++k) prefetch(k);
+        // paced by a counter, not by the barriers: a hint may fall behind or give up without harm
+        volatile int *progress = &bars.conv_progress;
+        for (int k = 0; k + kPrefetchAhead < my_steps; ++k) {
+            int done = *progress;
+            for (int polls = 0; done <= k && polls < (1 << 20) && !*abort_flag; ++polls) {
+                __nanosleep(100);
+                done = *progress;
+            }
+            if (done <= k) break;
+            k = done - 1;  // the newest finished step, should this warp have fallen behind
+            prefetch(k + kPrefetchAhead);
+        }
     } else if (warp < 4 || warp >= kFirstExtraConv) {
         // ------------------------------------------------------------------ converters
         // A step's operand block has at most 2 * kConvWarps row sets of 32 grid positions; warp cw
@@ -198,7 +241,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
         // the loads of the warp's next two sets travel (one set in flight exposes the full memory
         // latency per set).
         static_assert(kMmaWarps1 <= 4 && kConvWarps >= 1, "roles");
-        const int cw = warp < 4 ? warp - kMmaWarps1 : warp - kFirstExtraConv + (4 - kMmaWarps1);
+        const int cw = warp < 4 ? warp - kMmaWarps1 : warp - kFirstExtraConv + (4 - kMmaWarps1);  // 0 .. kConvWarps - 1
         const int step_rows = (T * S + 1) * Ws;            // grid positions a step's block holds
         const int W = ATARI ? 84 : p.in_w, plane = ATARI ? 84 * 84 : p.in_plane;
         const int posA = cw * 32 + lane, posB = (cw + kConvWarps) * 32 + lane;
@@ -251,7 +294,10 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
             load(wb, k + 1, RlB, XB, vB);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(full0 + 8 * s);
+            if (lane == 0) {
+                mbar_arrive(full0 + 8 * s);
+                if (cw == 0) *(volatile int *)&bars.conv_progress = k + 1;
+            }
         }
     } else {
         // ------------------------------------------------------------------ epilogue
