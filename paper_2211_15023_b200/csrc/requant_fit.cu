@@ -23,7 +23,7 @@ namespace accerl {
 
 namespace {
 
-constexpr int kKOffsets = 9;    // k2: 0, +1, -1, ... +4, -4 ulps
+constexpr int kKOffsets = 25;   // k2: 0, +1, -1, ... +12, -12 ulps
 constexpr int kBOffsets = 49;   // b2: 0, +1, -1, ... +24, -24 steps of 2^-21
 constexpr int kFitThreads = 256;
 constexpr int kPerThread = 16;  // accumulators a thread compares between two votes
