@@ -85,10 +85,9 @@ enum {
     ACCERL_FLAG_TEST_NO_FASTDIV = 16, /* test hook: treat every output scale as one for which the
                                          division-free requantiser could not be verified at create.
                                          Layers then run the epilogue that re-does elements near a
-                                         rounding tie with the IEEE divide, and plans that have no
-                                         such epilogue give way to the plain CUDA-core kernels --
-                                         what a policy with an unlucky scale gets.  Results are
-                                         the same bits either way. */
+                                         rounding tie with the IEEE divide -- what a policy with an
+                                         unlucky scale gets for that layer.  Results are the same
+                                         bits either way. */
     ACCERL_FLAG_TEST_NO_AFFINE = 32   /* test hook: do not search the single-fma requantiser
                                          constants at create (a layer for which the search finds
                                          none for some channel behaves like this): the epilogues

@@ -287,7 +287,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
 // on every other tile (two tiles are drained at a time, one per accumulator stage); inside a pair a
 // warp produces two of the row's four (pooled pixel, 16-channel piece) items, each from the
 // accumulators of pixels 2j .. 2j+2.
-template <bool RELU, bool AFFINE>
+template <bool RELU, int MODE>
 __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
 {
     const int q = warp & 3, wg = (warp - kProdWarps - kMmaWarps) >> 2;
@@ -346,8 +346,9 @@ __device__ __forceinline__ void epilogue_hpool(const TcGemmParams &p, const EpiC
                 bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
             }
             uint32_t w[4];
-            if (AFFINE) requant16_affine<RELU>(acc, ks, bs, w);
-            else requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+            if (MODE == kEpiAffine) requant16_affine<RELU>(acc, ks, bs, w);
+            else if (MODE == kEpiFastDiv) requant16_fastdiv<RELU>(acc, ks, bs, s_out, inv_s_out, w);
+            else requant16(acc, ks, bs, RELU, s_out, inv_s_out, w);
             if (row_ok && X * (4 / hpc) + ox < p.px_w)
                 *reinterpret_cast<uint4 *>(dst_row + ox * p.out_pitch + 16 * half) = make_uint4(w[0], w[1], w[2], w[3]);
         }
@@ -406,7 +407,10 @@ __device__ __forceinline__ void convert_tile(const TcGemmParams &p, const uint8_
 // FUSE is the first conv with the input stage inside (TcGemmParams::fuse_ingest).
 // PXK is the kernel for rows of several output pixels; it is kept apart so that its epilogue
 // variants do not weigh on the register allocation of the others.
-template <bool RESIDENT_B, bool EXTRAS, bool PXK, bool FUSE, bool AFFINE>
+// REQ: the requantiser of the launch's epilogue -- 0: three-step division (or, in the kernels without
+// multi-pixel rows, whatever the layer's switches say: logits, tie check), 1: single fma, 2: tie check
+// (multi-pixel rows whose output scale failed the division check)
+template <bool RESIDENT_B, bool EXTRAS, bool PXK, bool FUSE, int REQ>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const TcGemmParams p)
@@ -794,11 +798,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         asm volatile("griddepcontrol.wait;" ::: "memory");
         // (the requantiser is a template parameter of the kernel, not a branch: with both epilogues in
         // one kernel the layers measured slower)
-        constexpr int kDivFree = AFFINE ? kEpiAffine : kEpiFastDiv;
-        if constexpr (PXK) {  // multi-pixel rows: only built for the verified requantisers
+        constexpr bool AFFINE = REQ == 1;
+        constexpr int kDivFree = REQ == 1 ? kEpiAffine : (REQ == 2 ? kEpiTieCheck : kEpiFastDiv);
+        if constexpr (PXK) {  // multi-pixel rows: one requantiser per kernel
             if (p.hpool) {
-                if (p.relu_out) epilogue_hpool<true, AFFINE>(p, c, warp, lane);
-                else epilogue_hpool<false, AFFINE>(p, c, warp, lane);
+                if (p.relu_out) epilogue_hpool<true, kDivFree>(p, c, warp, lane);
+                else epilogue_hpool<false, kDivFree>(p, c, warp, lane);
             } else if (p.staged) {
                 if (p.relu_out) epilogue_role<EXTRAS, kDivFree, true, true, true, KS>(p, c, warp, lane);
                 else epilogue_role<EXTRAS, kDivFree, false, true, true, KS>(p, c, warp, lane);
@@ -978,22 +983,28 @@ cudaError_t tc_launch(const void *map_a, const void *map_b, const TcGemmParams &
     };
     cudaError_t e;
     if (p.affine && (!p.fast_div || p.logits_mode)) return cudaErrorInvalidValue;
-    auto pick = [&](auto affine) -> cudaError_t {
-        constexpr bool A = decltype(affine)::value;
-        if (p.px_per_row) {
-            if (!resident_b || !p.fast_div || p.logits_mode) return cudaErrorInvalidValue;
-            return extras ? go(tc_gemm_kernel<true, true, true, false, A>) : go(tc_gemm_kernel<true, false, true, false, A>);
+    auto pick = [&](auto req) -> cudaError_t {
+        constexpr int R = decltype(req)::value;
+        if constexpr (R == 2) {  // only the multi-pixel kernels have the tie check as a kernel of its own
+            if (!p.px_per_row || !resident_b || p.logits_mode) return cudaErrorInvalidValue;
+            return extras ? go(tc_gemm_kernel<true, true, true, false, 2>) : go(tc_gemm_kernel<true, false, true, false, 2>);
+        } else {
+            if (p.px_per_row) {
+                if (!resident_b || !p.fast_div || p.logits_mode) return cudaErrorInvalidValue;
+                return extras ? go(tc_gemm_kernel<true, true, true, false, R>) : go(tc_gemm_kernel<true, false, true, false, R>);
+            }
+            if (p.fuse_ingest) {
+                if (!resident_b || extras || !p.shifted || p.n_stages != p.n_mma) return cudaErrorInvalidValue;
+                return go(tc_gemm_kernel<true, false, false, true, R>);
+            }
+            return resident_b ? (extras ? go(tc_gemm_kernel<true, true, false, false, R>)
+                                        : go(tc_gemm_kernel<true, false, false, false, R>))
+                              : (extras ? go(tc_gemm_kernel<false, true, false, false, R>)
+                                        : go(tc_gemm_kernel<false, false, false, false, R>));
         }
-        if (p.fuse_ingest) {
-            if (!resident_b || extras || !p.shifted || p.n_stages != p.n_mma) return cudaErrorInvalidValue;
-            return go(tc_gemm_kernel<true, false, false, true, A>);
-        }
-        return resident_b ? (extras ? go(tc_gemm_kernel<true, true, false, false, A>)
-                                    : go(tc_gemm_kernel<true, false, false, false, A>))
-                          : (extras ? go(tc_gemm_kernel<false, true, false, false, A>)
-                                    : go(tc_gemm_kernel<false, false, false, false, A>));
     };
-    e = p.affine ? pick(std::true_type()) : pick(std::false_type());
+    e = p.affine ? pick(std::integral_constant<int, 1>())
+        : (p.px_per_row && !p.fast_div) ? pick(std::integral_constant<int, 2>()) : pick(std::integral_constant<int, 0>());
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

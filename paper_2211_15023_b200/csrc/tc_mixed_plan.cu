@@ -759,21 +759,13 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             }
         }
         g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first) || hp_out) ? 1 : 0;
-        if (role[i] == TCPX && !g.fast_div) {  // multi-pixel rows need the verified division
-            p->plan_note = "tensor-core plan not used: the division-free requantiser could not be verified for the "
-                           "output scale of layer " + std::to_string(i);
-            return bail();
-        }
+        // (a multi-pixel layer whose output scale fails the division check keeps its place in the plan:
+        // its launch runs the epilogue that re-does elements near a rounding tie with the IEEE divide)
         if (hp_out) {
             g.hpool = 1;
             g.px_w = (L.out_w - 3) / 2 + 1;  // pooled width
         }
         if (role[i] == TCFIRST && hpool_first) {
-            if (!g.fast_div) {
-                p->plan_note = "tensor-core plan not used: the division-free requantiser could not be verified for the "
-                               "output scale of layer " + std::to_string(i);
-                return bail();
-            }
             g.hpool = 1;
             g.px_per_row = 8;  // selects the multi-pixel kernel
             g.px_cols = d.out_c;
@@ -807,6 +799,7 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
         s.tc = (int)p->tc_steps.size() - 1;
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
         if (g.fast_div) s.kernel += g.affine ? "[single-fma requantiser verified]" : "[3-step divide verified]";
+        else if (!logits) s.kernel += "[division check failed: exact divide near ties]";
         if (g.hpool) s.kernel += "[pooled along x on the accumulators]";
         steps.push_back(s);
     }

@@ -632,6 +632,7 @@ accerl_status build_tc_plan(accerl_policy *p, const accerl_layer_desc *layers, i
         s.tc = (int)p->tc_steps.size() - 1;
         s.kernel = ts.resident_b ? "tc_gemm_kernel<resident weights>" : "tc_gemm_kernel<streamed weights>";
         if (g.fast_div) s.kernel += requant_note;
+        else if (!logits) s.kernel += "[division check failed: exact divide near ties]";
         s.covers = "layer " + std::to_string(i);
         if (g.fuse_ingest) {  // takes the place of the ingest launch
             s.kernel += "[frames quantised inside]";

@@ -456,10 +456,10 @@ def test_abi_rejects_bad_calls_without_launching():
 @pytest.mark.parametrize("name,b", [("nature_cnn_b160", 37), ("student_cnn_b8192", 21), ("impala_resnet_b16384", 5)])
 def test_policies_whose_output_scales_fail_the_division_check(name, b):
     """The create-time check of the division-free requantiser can reject an output scale.  With the
-    test flag every scale counts as rejected: the Nature-CNN plans then run the epilogue that redoes
-    elements near a rounding tie with the IEEE divide (still on tensor cores, input stage still
-    inside the first conv), the residual stacks fall back to the CUDA-core kernels and the plan
-    says why.  Bits must not change."""
+    test flag every scale counts as rejected: every layer then runs the epilogue that redoes
+    elements near a rounding tie with the IEEE divide -- still on tensor cores, the input stage
+    still inside the first conv of the Nature-CNN plans, the residual stacks still on their
+    multi-pixel rows and pooled accumulators -- and the plan says so.  Bits must not change."""
     import paper_2211_15023_b200 as P
     pol = calibrated(name, 64)
     obs, u = W.observations(name, b), W.uniforms(name, b)
@@ -468,10 +468,11 @@ def test_policies_whose_output_scales_fail_the_division_check(name, b):
         g = P.Policy(pol, b, flags=flags)
         plan = g.info()["plan"]
         assert "3-step divide verified" not in plan and "single-fma" not in plan, plan
+        assert "tc_gemm_kernel" in plan and "division check failed" in plan and "note:" not in plan, plan
         if name == "impala_resnet_b16384":
-            assert "note: tensor-core plan not used" in plan and "conv_dp4a_kernel" in plan, plan
+            assert "dp4a" not in plan and ("pooled along x on the accumulators" in plan or flags & 1), plan
         else:
-            assert "tc_gemm_kernel" in plan and "frames quantised inside" in plan, plan
+            assert "frames quantised inside" in plan, plan
         out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
         g.check()
         compare(ref, *out, taps=g.read_activation if flags & 1 else None)
