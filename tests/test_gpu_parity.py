@@ -504,3 +504,36 @@ def test_single_fma_requantiser_and_the_division_it_replaces_give_the_same_bits(
         compare(ref, *out, taps=g.read_activation if flags & 1 else None)
         g.close()
 
+
+@pytest.mark.parametrize("case", ["coarse_scale", "fine_scale", "bias_far_below", "bias_far_above", "tiny_weight_scale"])
+def test_requantiser_constants_at_the_edges_of_their_search(case):
+    """The band of accumulators the single-fma constants are checked on comes from the layer's
+    scales and biases.  Scales and biases far from what calibration gives (every output saturated,
+    every output in a handful of codes, bands that touch the int32 limits) must either find
+    constants that still equal the defining expression or leave the layer on the division; the
+    oracle decides, tensor by tensor, with and without the search."""
+    import copy
+    import paper_2211_15023_b200 as P
+    name, b = "student_cnn_b8192", 33
+    pol = copy.deepcopy(calibrated(name, 64))
+    l1, l2 = pol["layers"][1], pol["layers"][2]
+    if case == "coarse_scale":          # nearly everything rounds to -1, 0 or 1
+        l1["s_out"] = np.float32(l1["s_out"] * 90.0)
+    elif case == "fine_scale":          # nearly everything saturates
+        l1["s_out"] = np.float32(l1["s_out"] / 500.0)
+    elif case == "bias_far_below":      # ReLU leaves zeros only
+        l1["bias"] = (l1["bias"] - np.float32(1000.0) * l1["s_out"]).astype(np.float32)
+    elif case == "bias_far_above":      # every code is 127
+        l1["bias"] = (l1["bias"] + np.float32(1000.0) * l1["s_out"]).astype(np.float32)
+    else:                               # a band of accumulators wider than int32
+        l1["s_w"] = (l1["s_w"] * np.float32(1e-7)).astype(np.float32)
+    l2["s_in"] = l1["s_out"]
+    obs, u = W.observations(name, b), W.uniforms(name, b)
+    ref = oracle.forward(pol, obs, u)
+    for flags in (1, 0, 1 | P.FLAG_TEST_NO_AFFINE):
+        g = P.Policy(pol, b, flags=flags)
+        out = [t.cpu().numpy() for t in g.act(torch.from_numpy(obs).cuda(), torch.from_numpy(u).cuda())]
+        g.check()
+        compare(ref, *out, taps=g.read_activation if flags & 1 else None)
+        g.close()
+
