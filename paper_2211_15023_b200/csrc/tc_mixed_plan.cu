@@ -747,18 +747,9 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
             volatile float inv = 1.0f / L.s_out;
             g.inv_s_out = inv;
         }
-        if (!logits) {
-            float kmax = 0.f, bmax = 0.f;
-            for (int c = 0; c < d.out_c; ++c) {
-                kmax = std::max(kmax, d.s_in * d.s_w[c]);
-                bmax = std::max(bmax, fabsf(d.bias[c]));
-            }
-            st = choose_fastdiv(g.s_out, g.relu_out != 0, 2147483648.0f * kmax + bmax,
-                                !(p->flags & ACCERL_FLAG_TEST_NO_FASTDIV), &g.inv_s_out, &g.fast_div);
-            if (st != ACCERL_OK) return st;
-        }
-        // the single-fma requantiser where every channel has verified constants
-        if (!logits && g.fast_div && !(p->flags & ACCERL_FLAG_TEST_NO_AFFINE)) {
+        // the single-fma requantiser where every channel has verified constants (searched first: a layer
+        // that has them needs no check of the three-step division)
+        if (!logits && !(p->flags & ACCERL_FLAG_TEST_NO_FASTDIV) && !(p->flags & ACCERL_FLAG_TEST_NO_AFFINE)) {
             const bool repeated = role[i] == TCFIRST || P;  // columns = (pixel of the row, channel)
             std::vector<float> kh(n_total, 0.f), bh(n_total, 0.f), k2, b2;
             for (int j = 0; j < n_total; ++j) {
@@ -778,7 +769,18 @@ accerl_status build_tc_mixed_plan(accerl_policy *p, const accerl_layer_desc *lay
                 g.kscale = (const float *)kd;
                 g.bias = (const float *)bd;
                 g.affine = 1;
+                g.fast_div = 1;  // a verified division-free requantiser exists
             }
+        }
+        if (!logits && !g.affine) {
+            float kmax = 0.f, bmax = 0.f;
+            for (int c = 0; c < d.out_c; ++c) {
+                kmax = std::max(kmax, d.s_in * d.s_w[c]);
+                bmax = std::max(bmax, fabsf(d.bias[c]));
+            }
+            st = choose_fastdiv(g.s_out, g.relu_out != 0, 2147483648.0f * kmax + bmax,
+                                !(p->flags & ACCERL_FLAG_TEST_NO_FASTDIV), &g.inv_s_out, &g.fast_div);
+            if (st != ACCERL_OK) return st;
         }
         g.split_cols = (g.n_tile > 128 || (role[i] == TCFIRST && hpool_first) || hp_out) ? 1 : 0;
         // (a multi-pixel layer whose output scale fails the division check keeps its place in the plan:
