@@ -198,12 +198,15 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const float s_out = p.s_out, inv_s_out = p.inv_s_out;
         asm volatile("griddepcontrol.wait;" ::: "memory");  // the output may reuse a buffer an earlier launch reads
         bool ok = true;
-        for (int k = 0; k < my_steps && ok; ++k) {
-            const int step = (int)blockIdx.x + k * (int)gridDim.x;
-            for (int i = 0; i < T; ++i) {
-                const int tile = step * T + i, seq = k * T + i;  // seq: the CTA's tiles in order
-                if (tile >= p.total_tiles) break;
-                if (seq % kGroups != wg) continue;
+        // warpgroup wg takes the CTA's tiles wg, wg + kGroups, ... (seq: the CTA's tiles in order;
+        // T is 1, 2 or 4)
+        const int t_log2 = T == 4 ? 2 : (T == 2 ? 1 : 0);
+        for (int seq = wg; ok; seq += kGroups) {
+            {
+                const int k = seq >> t_log2, i = seq & (T - 1);
+                if (k >= my_steps) break;
+                const int tile = ((int)blockIdx.x + k * (int)gridDim.x) * T + i;
+                if (tile >= p.total_tiles) break;  // only the last step is short, and later tiles lie behind it
                 const int slot = seq % kAccSlots;
                 ok = mbar_wait(acc_full0 + 8 * slot, (uint32_t)((seq / kAccSlots) & 1), abort_flag, p.status, 16);
                 ok = __all_sync(0xffffffffu, ok);
