@@ -237,9 +237,11 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         if (32 * hh + 16 * h >= NCOLS) continue;
                         float ks[16], bs[16];
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) {  // kernel parameters: read from the constant bank
-                            ks[e] = p.ks[32 * hh + 16 * h + e];
-                            bs[e] = p.bs[32 * hh + 16 * h + e];
+                        for (int g = 0; g < 4; ++g) {  // kernel parameters: 16-byte reads from the constant bank
+                            const float4 kv = *reinterpret_cast<const float4 *>(&p.ks[32 * hh + 16 * h + 4 * g]);
+                            const float4 bv = *reinterpret_cast<const float4 *>(&p.bs[32 * hh + 16 * h + 4 * g]);
+                            ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                            bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
                         }
                         uint32_t wv[4];
                         if (AFFINE) {

@@ -24,7 +24,7 @@ struct ConvRowsParams {
     float s_out, inv_s_out;
     int relu;
     int affine;                      // 1: ks / bs are the single-fma constants (k2, b2)
-    float ks[64], bs[64];            // s_in * s_w[c] and bias per output channel
+    alignas(16) float ks[64], bs[64];            // s_in * s_w[c] and bias per output channel
     int *status;
 };
 

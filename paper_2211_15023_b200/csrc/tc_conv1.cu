@@ -344,9 +344,11 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 for (int h = 0; h < NCOLS / 16; ++h) {
                     float ks[16], bs[16];
 #pragma unroll
-                    for (int e = 0; e < 16; ++e) {  // kernel parameters: read from the constant bank
-                        ks[e] = p.ks[16 * h + e];
-                        bs[e] = p.bs[16 * h + e];
+                    for (int g = 0; g < 4; ++g) {  // kernel parameters: 16-byte reads from the constant bank
+                        const float4 kv = *reinterpret_cast<const float4 *>(&p.ks[16 * h + 4 * g]);
+                        const float4 bv = *reinterpret_cast<const float4 *>(&p.bs[16 * h + 4 * g]);
+                        ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
+                        bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
                     }
                     uint32_t wv[4];
                     if (AFFINE) {

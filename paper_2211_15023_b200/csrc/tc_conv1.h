@@ -26,7 +26,7 @@ struct Conv1Params {
     float s_out, inv_s_out;
     int relu;
     int affine;                      // 1: ks / bs are the single-fma constants (k2, b2)
-    float ks[32], bs[32];            // s_in * s_w[c] and bias per output channel
+    alignas(16) float ks[32], bs[32];            // s_in * s_w[c] and bias per output channel
     int *status;
 };
 
