@@ -265,19 +265,26 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 for (int dy = 0; dy < 4; ++dy)
                     w[4 * c + dy] = __ldg(reinterpret_cast<const uint32_t *>(src + (size_t)c * plane + dy * W));
         };
-        // quantise one set and write its operand rows (16-byte pieces under the 64-byte swizzle)
-        auto store = [&](const uint32_t (&w)[16], uint8_t *block, int pos, bool v) {
+        // quantise one set and write its operand rows: four 16-byte pieces under the 64-byte swizzle,
+        // at 32-bit shared-memory addresses whose per-thread parts (off[c]) are computed once
+        auto store = [&](const uint32_t (&w)[16], uint32_t block, const uint32_t (&off)[4], bool v) {
             if (!v) return;
-            uint8_t *row = block + pos * 64;
-            const int sw = (pos >> 1) & 3;
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-                *reinterpret_cast<uint4 *>(row + ((c ^ sw) << 4)) =
-                    make_uint4(quantise_word<MODE>(w[4 * c], p.ingest_mul, p.ingest_add),
-                               quantise_word<MODE>(w[4 * c + 1], p.ingest_mul, p.ingest_add),
-                               quantise_word<MODE>(w[4 * c + 2], p.ingest_mul, p.ingest_add),
-                               quantise_word<MODE>(w[4 * c + 3], p.ingest_mul, p.ingest_add));
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(block + off[c]),
+                             "r"(quantise_word<MODE>(w[4 * c], p.ingest_mul, p.ingest_add)),
+                             "r"(quantise_word<MODE>(w[4 * c + 1], p.ingest_mul, p.ingest_add)),
+                             "r"(quantise_word<MODE>(w[4 * c + 2], p.ingest_mul, p.ingest_add)),
+                             "r"(quantise_word<MODE>(w[4 * c + 3], p.ingest_mul, p.ingest_add))
+                             : "memory");
         };
+        uint32_t offA[4], offB[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            offA[c] = (uint32_t)(posA * 64 + ((c ^ ((posA >> 1) & 3)) << 4));
+            offB[c] = (uint32_t)(posB * 64 + ((c ^ ((posB >> 1) & 3)) << 4));
+        }
+        const uint32_t stages_s = smem_u32(stages);
         uint32_t wa[16], wb[16];
         load(wa, 0, RlA, XA, vA);
         load(wb, 0, RlB, XB, vB);
@@ -287,10 +294,10 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
             ok = mbar_wait(empty0 + 8 * s, (uint32_t)(((k / kStages) & 1) ^ 1), abort_flag, p.status, 1);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            uint8_t *block = stages + (size_t)s * stage_bytes;
-            store(wa, block, posA, vA);
+            const uint32_t block = stages_s + (uint32_t)(s * stage_bytes);
+            store(wa, block, offA, vA);
             load(wa, k + 1, RlA, XA, vA);
-            store(wb, block, posB, vB);
+            store(wb, block, offB, vB);
             load(wb, k + 1, RlB, XB, vB);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
