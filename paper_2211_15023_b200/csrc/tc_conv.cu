@@ -217,8 +217,9 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const unsigned n = __umulhi(R, p.hs_magic);
                 const int Y = (int)(R - n * (unsigned)Hs);
                 const bool valid = row_ok && Y < p.out_h && (int)n < p.batch;
-                int8_t *dst = p.out + ((size_t)n * p.out_rows_per_image + (size_t)(Y >> sh) * p.out_grid_w) * p.out_pitch +
-                              ((Y & smask) << sh) * p.n_total + x_off;
+                int8_t *dst = p.out + (size_t)(n * (unsigned)p.out_rows_per_image + (unsigned)((Y >> sh) * p.out_grid_w)) *
+                                          (size_t)p.out_pitch +
+                              (((Y & smask) << sh) * p.n_total + x_off);
                 constexpr int kHalves = (NCOLS + 31) / 32;  // 32 columns at a time
 #pragma unroll
                 for (int hh = 0; hh < kHalves; ++hh) {

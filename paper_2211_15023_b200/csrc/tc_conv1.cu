@@ -253,12 +253,12 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
         // the last step reads the first image's bytes instead (its row is no output), which takes the
         // sixteen selects out of the loop (86 against 89.5 us for the layer)
         auto load = [&](uint32_t (&w)[16], int k, int Rl, int X, bool v) {
-            const int step = (int)blockIdx.x + k * (int)gridDim.x;
-            const long long R = (long long)step * (T * S) + Rl;
-            const bool in = v && k < my_steps && R < p.total_grid_rows;
-            const unsigned n = div_hs((unsigned)R);
-            const int Y = (int)((unsigned)R - n * (unsigned)Hs);
-            const uint8_t *src = p.obs + (in ? (size_t)n * 4 * plane + (size_t)(4 * Y) * W + 4 * X : (size_t)0);
+            // (32-bit row arithmetic: the plan has checked that batch * grid_h + 64 < 2^31)
+            const unsigned R = (unsigned)(((int)blockIdx.x + k * (int)gridDim.x) * (T * S) + Rl);
+            const bool in = v && k < my_steps && R < (unsigned)p.total_grid_rows;
+            const unsigned n = div_hs(R);
+            const int Y = (int)(R - n * (unsigned)Hs);
+            const uint8_t *src = p.obs + (in ? (size_t)n * (size_t)(4 * plane) + (size_t)(4 * Y * W + 4 * X) : (size_t)0);
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -345,8 +345,9 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 const unsigned n = div_hs(R);
                 const int Y = (int)(R - n * (unsigned)Hs);
                 const bool valid = row_ok && Y < p.out_h && (int)n < p.batch;
-                int8_t *dst = p.out + ((size_t)n * p.out_rows_per_image + (size_t)(Y >> sh) * p.out_grid_w) * p.out_pitch +
-                              ((Y & smask) << sh) * p.n_total + x_off;
+                int8_t *dst = p.out + (size_t)(n * (unsigned)p.out_rows_per_image + (unsigned)((Y >> sh) * p.out_grid_w)) *
+                                          (size_t)p.out_pitch +
+                              (((Y & smask) << sh) * p.n_total + x_off);
 #pragma unroll
                 for (int h = 0; h < NCOLS / 16; ++h) {
                     float ks[16], bs[16];
@@ -410,7 +411,7 @@ bool conv1_plan(const accerl_layer_desc &d, int in_h, int in_w, long long max_ba
     const int S = 128 / Ws;
     if (S * Ws < 112) return false;  // too many idle rows per tile
     const long long rows = max_batch * Hs;
-    if (rows + 64 >= (1LL << 31)) return false;
+    if (rows + 64 >= (1LL << 31) || rows * Ws >= (1LL << 31)) return false;  // 32-bit row and output-row indices
     memset(q, 0, sizeof(*q));
     if (!magic_exact((unsigned)Ws, (unsigned long long)(kMaxT * S + 2) * Ws + 64, &q->ws_magic)) return false;
     if (!magic_exact((unsigned)Hs, (unsigned long long)rows + 256, &q->hs_magic)) return false;
