@@ -81,6 +81,18 @@ constexpr int kStagingBytes = 32 * 128;  // 32 rows of 128 output bytes
 // warp's pieces over the banks both when lanes are rows and when eight lanes share a row
 __device__ __forceinline__ int stage_off(int row, int ch) { return row * 128 + ((ch ^ (row & 7)) << 4); }
 
+// 16-byte accesses to a warp's staging tile at 32-bit shared-memory addresses
+__device__ __forceinline__ void sts16(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
 __device__ __forceinline__ uint4 relu_codes(uint4 v)
 {
     uint32_t w[4] = {v.x, v.y, v.z, v.w};
@@ -102,7 +114,7 @@ __device__ __forceinline__ uint4 relu_codes(uint4 v)
 template <bool EXTRAS, int MODE, bool RELU, bool PX, bool STAGED, bool KS>
 __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCtx &c, int warp, int lane)
 {
-    uint8_t *stage = STAGED ? c.staging + (warp - kProdWarps - kMmaWarps) * kStagingBytes : nullptr;
+    const uint32_t stage = STAGED ? smem_u32(c.staging + (warp - kProdWarps - kMmaWarps) * kStagingBytes) : 0u;
     const int q = warp & 3;         // this warp's quarter of tensor memory
     const int wg = (warp - kProdWarps - kMmaWarps) >> 2;  // epilogue warpgroup
     const int c_span = p.split_cols ? p.n_tile / kEpiGroups : p.n_tile;
@@ -187,7 +199,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                         const int np = __shfl_sync(0xffffffffu, my_pieces, r);
                         uint4 v = make_uint4(0, 0, 0, 0);
                         if (ch < np) v = __ldg(reinterpret_cast<const uint4 *>(p.skip) + so + ch);
-                        *reinterpret_cast<uint4 *>(stage + stage_off(r, ch)) = v;
+                        sts16(stage + (uint32_t)stage_off(r, ch), v);
                     }
                     __syncwarp();
                 }
@@ -215,7 +227,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 }
                 if (EXTRAS && has_skip) {  // residual add in the int32 domain
                     uint4 sv = make_uint4(0, 0, 0, 0);
-                    if (STAGED) sv = *reinterpret_cast<const uint4 *>(stage + stage_off(lane, c0 >> 4));
+                    if (STAGED) sv = lds16(stage + (uint32_t)stage_off(lane, c0 >> 4));
                     else if (valid && c0 < n_store) sv = __ldg(reinterpret_cast<const uint4 *>(skip + c0));
                     const uint32_t sw[4] = {sv.x, sv.y, sv.z, sv.w};
 #pragma unroll
@@ -245,7 +257,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                 else requant16(acc, ks, bs, RELU, s_out, inv_s_out, w);
                 const uint4 plain = make_uint4(w[0], w[1], w[2], w[3]);
                 if (STAGED) {
-                    *reinterpret_cast<uint4 *>(stage + stage_off(lane, c0 >> 4)) = plain;
+                    sts16(stage + (uint32_t)stage_off(lane, c0 >> 4), plain);
                 } else if (EXTRAS) {
                     uint4 relu = plain;
                     if (p.out_relu | p.out2_relu) {
@@ -270,7 +282,7 @@ __device__ __forceinline__ void epilogue_role(const TcGemmParams &p, const EpiCt
                     const uint32_t o = __shfl_sync(0xffffffffu, my_out16, r);
                     const uint32_t o2 = has_out2 ? __shfl_sync(0xffffffffu, my_out2_16, r) : 0u;
                     const int np = __shfl_sync(0xffffffffu, my_pieces, r);
-                    const uint4 v = *reinterpret_cast<const uint4 *>(stage + stage_off(r, ch));
+                    const uint4 v = lds16(stage + (uint32_t)stage_off(r, ch));
                     if (ch < np) {
                         const uint4 vr = (EXTRAS && (p.out_relu | p.out2_relu)) ? relu_codes(v) : v;
                         reinterpret_cast<uint4 *>(p.out)[o + ch] = (EXTRAS && p.out_relu) ? vr : v;
