@@ -112,7 +112,8 @@ bool make_job(float k, float b, float s_out, bool relu, FitJob *job)
     job->check_hi = hi <= 2147483647.0;
     job->lo = (long long)std::max(lo, -2147483648.0);
     job->hi = (long long)std::min(hi, 2147483647.0);
-    return job->hi >= job->lo && job->hi - job->lo <= (1LL << 27);
+    // (bands of the networks here have 65 k - 350 k accumulators; the limit bounds the search time)
+    return job->hi >= job->lo && job->hi - job->lo <= (1LL << 22);
 }
 
 }  // namespace
