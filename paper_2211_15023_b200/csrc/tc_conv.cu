@@ -233,6 +233,7 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         __syncwarp();
                         if (lane == 0) mbar_arrive(acc_empty0 + 8 * slot);
                     }
+                    uint32_t wq[kPieces][4];
 #pragma unroll
                     for (int h = 0; h < kPieces; ++h) {
                         if (32 * hh + 16 * h >= NCOLS) continue;
@@ -244,7 +245,7 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
                             bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
                         }
-                        uint32_t wv[4];
+                        uint32_t (&wv)[4] = wq[h];
                         if (AFFINE) {
                             if (p.relu) requant16_affine<true>(acc[h], ks, bs, wv);
                             else requant16_affine<false>(acc[h], ks, bs, wv);
@@ -252,7 +253,17 @@ conv_rows_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                             if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
                             else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
                         }
-                        if (valid) *reinterpret_cast<uint4 *>(dst + 32 * hh + 16 * h) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                    }
+                    if (valid) {  // 32 channels in one store where the channel count is a multiple of 32
+                        if constexpr (NCOLS % 32 == 0) {  // positions are then 32-byte aligned
+                            stg32(dst + 32 * hh, wq[0], wq[1]);
+                        } else {
+#pragma unroll
+                            for (int h = 0; h < kPieces; ++h)
+                                if (32 * hh + 16 * h < NCOLS)
+                                    *reinterpret_cast<uint4 *>(dst + 32 * hh + 16 * h) =
+                                        make_uint4(wq[h][0], wq[h][1], wq[h][2], wq[h][3]);
+                        }
                     }
                 }
             }

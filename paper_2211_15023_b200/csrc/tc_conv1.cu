@@ -348,6 +348,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                 int8_t *dst = p.out + (size_t)(n * (unsigned)p.out_rows_per_image + (unsigned)((Y >> sh) * p.out_grid_w)) *
                                           (size_t)p.out_pitch +
                               (((Y & smask) << sh) * p.n_total + x_off);
+                uint32_t wq[NCOLS / 16][4];
 #pragma unroll
                 for (int h = 0; h < NCOLS / 16; ++h) {
                     float ks[16], bs[16];
@@ -358,7 +359,7 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                         ks[4 * g] = kv.x; ks[4 * g + 1] = kv.y; ks[4 * g + 2] = kv.z; ks[4 * g + 3] = kv.w;
                         bs[4 * g] = bv.x; bs[4 * g + 1] = bv.y; bs[4 * g + 2] = bv.z; bs[4 * g + 3] = bv.w;
                     }
-                    uint32_t wv[4];
+                    uint32_t (&wv)[4] = wq[h];
                     if (AFFINE) {
                         if (p.relu) requant16_affine<true>(acc[h], ks, bs, wv);
                         else requant16_affine<false>(acc[h], ks, bs, wv);
@@ -366,7 +367,10 @@ conv1_frames_kernel(const __grid_constant__ CUtensorMap map_b, const __grid_cons
                         if (p.relu) requant16_fastdiv<true>(acc[h], ks, bs, s_out, inv_s_out, wv);
                         else requant16_fastdiv<false>(acc[h], ks, bs, s_out, inv_s_out, wv);
                     }
-                    if (valid) *reinterpret_cast<uint4 *>(dst + 16 * h) = make_uint4(wv[0], wv[1], wv[2], wv[3]);
+                }
+                if (valid) {  // a position's channels are contiguous: 16 bytes, or 32 in one store
+                    if constexpr (NCOLS == 32) stg32(dst, wq[0], wq[1]);
+                    else *reinterpret_cast<uint4 *>(dst) = make_uint4(wq[0][0], wq[0][1], wq[0][2], wq[0][3]);
                 }
             }
         }

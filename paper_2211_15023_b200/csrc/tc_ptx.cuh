@@ -154,6 +154,15 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&r)[16])
         : "memory");
 }
 
+// one 32-byte store (the address a multiple of 32): half the load/store wavefronts of two 16-byte
+// stores whose lanes are 32 bytes apart
+__device__ __forceinline__ void stg32(void *dst, const uint32_t (&a)[4], const uint32_t (&b)[4])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(a[0]), "r"(a[1]), "r"(a[2]),
+                 "r"(a[3]), "r"(b[0]), "r"(b[1]), "r"(b[2]), "r"(b[3])
+                 : "memory");
+}
+
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int (&r)[32])
 {
     asm volatile(
