@@ -189,12 +189,12 @@ def algorithmic(name: str, batch: int) -> dict:
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch / states of that launch, from
-# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 173.47 MB read + 48.26 MB written by the
+# profiles/ncu_full_nature_cnn_b6144.md (batch 6144: 173.47 MB read + 50.96 MB written by the
 # first conv with the input stage inside)
 _CONV1 = "conv1_frames_kernel[single-fma requantiser verified][frames quantised inside]"
-NCU_DRAM_BYTES_PER_STATE = {("nature_cnn_b8192", _CONV1): (173470208 + 48264192) / 6144}
+NCU_DRAM_BYTES_PER_STATE = {("nature_cnn_b8192", _CONV1): (173472000 + 50957824) / 6144}
 # warp-level instructions executed per state by the dominant kernel, from the same capture
-NCU_WARP_INST_PER_STATE = {("nature_cnn_b8192", _CONV1): 30467423 / 6144}
+NCU_WARP_INST_PER_STATE = {("nature_cnn_b8192", _CONV1): 28499170 / 6144}
 
 
 def launch_work(name: str, plan: str, batch: int) -> list:
